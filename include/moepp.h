@@ -1,0 +1,177 @@
+/*
+ * moepp.h -- C ABI of the MoE++ heterogeneous expert layer (forward pass) for NVIDIA B200 (sm_100a).
+ *
+ * The layer is the one defined in "MoE++: Accelerating Mixture-of-Experts Methods with
+ * Zero-Computation Experts" (arXiv 2410.07348):
+ *   Eq. 1  y = sum_i g_i E_i(x),  g_i = Softmax(G(x))_i if i is among the Top-K logits, else 0
+ *   Eq. 2  vanilla router G(x) = W x
+ *   Eq. 3  zero expert      E(x) = 0
+ *   Eq. 4  copy expert      E(x) = x
+ *   Eq. 5  constant expert  E(x) = a1 x + a2 v,  [a1, a2] = Softmax(W_c x)
+ *   Eq. 6  gating residual  G(x^j) = W^j x^j + W_g^j G(x^{j-1})   (first layer: no residual term)
+ * FFN experts are bias-free SwiGLU networks: W_down (silu(W_gate x) * (W_up x)).
+ *
+ * Conventions shared by every call
+ *   - All pointers are DEVICE pointers owned by the caller unless a parameter says "host".
+ *     The library allocates nothing and frees nothing.  Work is enqueued on `stream`
+ *     (a cudaStream_t passed as void*; NULL = the default stream) and the call returns
+ *     without synchronising.
+ *   - Row-major everywhere.  T tokens, D model width, F FFN width, K = top_k,
+ *     N = n_ffn + n_zero + n_copy + n_const experts, indexed in that order
+ *     (FFN | zero | copy | constant).  Slot s = t*K + k is the k-th pick of token t.
+ *   - `dtype` is the storage type of x, y, x_perm, h, y_perm and the FFN weights.
+ *     Router weights, logits, gate weights, W_c, v and all accumulation are float.
+ *   - Activation and FFN-weight pointers must be 16-byte aligned; D and F must be
+ *     multiples of 8 (MOEPP_ERR_ALIGN otherwise).
+ *   - M_cap = T*K + n_ffn*(row_align-1) is the row capacity of the grouped buffers.
+ *   - Errors are returned, never thrown: argument errors are found on the host before
+ *     anything is launched; MOEPP_ERR_CUDA wraps a failed launch.  T == 0 is valid and does nothing.
+ *   - Limits: N <= 64, 1 <= K <= min(N, 8), N + 2*n_const <= 128.
+ */
+#ifndef MOEPP_H
+#define MOEPP_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  MOEPP_OK = 0,
+  MOEPP_ERR_INVALID_ARG = 1,
+  MOEPP_ERR_UNSUPPORTED = 2,
+  MOEPP_ERR_ALIGN = 3,
+  MOEPP_ERR_WORKSPACE = 4,
+  MOEPP_ERR_CUDA = 5,
+  MOEPP_ERR_TIMEOUT = 6
+} moepp_status;
+
+typedef enum { MOEPP_F32 = 0, MOEPP_BF16 = 1 } moepp_dtype;
+
+/* flags */
+#define MOEPP_FLAG_LOGITS_GIVEN 1 /* moepp_route reads `logits` instead of computing Eq. 2 / Eq. 6 */
+#define MOEPP_FLAG_SIMT_FFN 2     /* bf16 only: run the FFN on the plain FMA kernel (cross-check path) */
+
+typedef struct {
+  int32_t T, D, F;
+  int32_t n_ffn, n_zero, n_copy, n_const; /* expert index order: FFN | zero | copy | constant */
+  int32_t top_k;                          /* the paper uses 2 in every layer */
+  int32_t dtype;                          /* moepp_dtype */
+  int32_t renorm_topk;                    /* 0: Eq. 1 as printed; 1: divide the K gate weights by their sum */
+  int32_t row_align;                      /* 1: dense grouped layout; >1: pad each expert's rows to a multiple */
+  int32_t add_residual;                   /* 0: y is Eq. 1; 1: y = x + Eq. 1 (for stacking layers) */
+  int32_t flags;                          /* MOEPP_FLAG_* */
+} moepp_config;
+
+typedef struct {
+  const float* W_r;         /* [N, D]            Eq. 2 / Eq. 6 */
+  const float* W_g;         /* [N, N] or NULL    Eq. 6 */
+  const float* W_c;         /* [n_const, 2, D]   Eq. 5 (each constant expert has its own) */
+  const float* v;           /* [n_const, D]      Eq. 5 */
+  const float* router_bias; /* [N] or NULL; not part of the method, only shapes the load in benchmarks */
+  const void* W_gate;       /* [n_ffn, F, D] */
+  const void* W_up;         /* [n_ffn, F, D] */
+  const void* W_down;       /* [n_ffn, D, F] */
+} moepp_weights;
+
+const char* moepp_status_string(moepp_status s);
+
+/* Bytes of device scratch moepp_layer_forward needs for this configuration (a pure host computation). */
+moepp_status moepp_workspace_bytes(const moepp_config* cfg, size_t* bytes);
+
+/*
+ * Router (Eq. 2, Eq. 6), gate (Eq. 1) and, if alpha is wanted, the constant experts' mixing weights (Eq. 5).
+ *   logits[t,i] = W_r[i,:].x[t,:] (+ W_g[i,:].prev_logits[t,:]) (+ router_bias[i])
+ *   P = softmax(logits[t,:]) over all N; the K largest logits are picked, larger first, equal
+ *   logits -> lower index first; topk_w = P at the picks (divided by their sum if renorm_topk).
+ *   expert_counts[e] = number of slots routed to e (all N experts);
+ *   expert_offsets[e] = first grouped row of FFN expert e, expert_offsets[n_ffn] = rows in use;
+ *   each expert's segment is its count rounded up to row_align.
+ * W_g and prev_logits are both NULL (first layer) or both set.  alpha may be NULL (then W_c is unused).
+ * With MOEPP_FLAG_LOGITS_GIVEN `logits` is an input and W_r, W_g, prev_logits, router_bias are ignored.
+ */
+moepp_status moepp_route(const moepp_config* cfg, const void* x, const float* W_r, const float* W_g,
+                         const float* prev_logits, const float* router_bias, const float* W_c,
+                         float* logits,           /* [T, N] out (in with MOEPP_FLAG_LOGITS_GIVEN) */
+                         int32_t* topk_idx,       /* [T, K] out */
+                         float* topk_w,           /* [T, K] out */
+                         int32_t* expert_counts,  /* [N] out */
+                         int32_t* expert_offsets, /* [n_ffn + 1] out */
+                         float* alpha,            /* [T, n_const, 2] out, or NULL */
+                         void* stream);
+
+/*
+ * Grouping of the FFN slots only; zero-computation slots get no row (the efficiency argument of the
+ * paper's Section 3.4 made literal).  Rows are expert-major and, inside an expert, ascend in slot id.
+ *   row_of_slot[s] = grouped row of slot s, or -1 for a zero-computation slot
+ *   slot_of_row[r] = slot held by row r, or -1 for a pad row / a row beyond expert_offsets[n_ffn]
+ *   x_perm[r,:]    = x[slot_of_row[r] / K, :]; pad rows inside a segment are zero-filled; rows at or
+ *                    beyond expert_offsets[n_ffn] are left untouched.
+ */
+moepp_status moepp_permute(const moepp_config* cfg, const void* x, const int32_t* topk_idx,
+                           const int32_t* expert_offsets,
+                           int32_t* row_of_slot, /* [T, K] out */
+                           int32_t* slot_of_row, /* [M_cap] out */
+                           void* x_perm,         /* [M_cap, D] out */
+                           void* stream);
+
+/*
+ * Grouped SwiGLU FFN: for each FFN expert e and each row r in [expert_offsets[e], expert_offsets[e+1])
+ *   h[r,:] = silu(W_gate[e] x_perm[r,:]) * (W_up[e] x_perm[r,:]);  y_perm[r,:] = W_down[e] h[r,:].
+ * bf16: tcgen05 tensor-core kernels fed by TMA, float accumulation in tensor memory, h and y_perm
+ * rounded once to bf16.  f32: FMA kernels.  h_ws is caller-provided scratch of M_cap*F elements.
+ */
+moepp_status moepp_grouped_ffn(const moepp_config* cfg, const void* x_perm, const int32_t* expert_offsets,
+                               const void* W_gate, const void* W_up, const void* W_down,
+                               void* h_ws,   /* [M_cap, F] scratch */
+                               void* y_perm, /* [M_cap, D] out */
+                               void* stream);
+
+/*
+ * Weighted combine (Eq. 1) with the zero-computation experts applied in place:
+ *   y[t,:] = (x[t,:] if add_residual) + sum_k topk_w[t,k] * c(t,k),
+ *   c = y_perm[row_of_slot[t,k],:] (FFN) | 0 (Eq. 3) | x[t,:] (Eq. 4) | a1 x[t,:] + a2 v[q,:] (Eq. 5).
+ * alpha may be NULL; the mixing weights are then computed here from W_c and x.
+ */
+moepp_status moepp_combine(const moepp_config* cfg, const void* x, const void* y_perm, const int32_t* topk_idx,
+                           const float* topk_w, const int32_t* row_of_slot,
+                           const float* alpha, /* [T, n_const, 2] or NULL */
+                           const float* W_c, const float* v,
+                           void* y, /* [T, D] out */
+                           void* stream);
+
+/*
+ * One whole layer: route -> permute -> grouped FFN -> combine, on one stream, without host
+ * synchronisation.  prev_logits is NULL for the first layer (then W_g must be NULL too).
+ * logits_out ([T, N], may be NULL) receives this layer's logits for the next layer's Eq. 6.
+ * workspace: device scratch of at least moepp_workspace_bytes(), 256-byte aligned.
+ */
+moepp_status moepp_layer_forward(const moepp_config* cfg, const moepp_weights* weights, const void* x,
+                                 const float* prev_logits, void* y, float* logits_out, void* workspace,
+                                 size_t workspace_bytes, void* stream);
+
+/*
+ * The same layer for a caller whose activations live in HOST memory (pinned memory for the copies
+ * to be asynchronous): x_host, prev_logits_host (or NULL), y_host and logits_out_host (or NULL) are
+ * host pointers; weights and workspace stay on the device.  The workspace must be
+ * moepp_workspace_bytes_host() large; copies and kernels are enqueued on `stream`, and the host
+ * buffers are valid once the stream has been synchronised.
+ */
+moepp_status moepp_workspace_bytes_host(const moepp_config* cfg, size_t* bytes);
+moepp_status moepp_layer_forward_host(const moepp_config* cfg, const moepp_weights* weights, const void* x_host,
+                                      const float* prev_logits_host, void* y_host, float* logits_out_host,
+                                      void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Device-side waits in the tensor-core kernels are bounded.  If one ever runs out, the kernel
+ * stops early and records a non-zero code; this call copies the code to *code (host pointer),
+ * clears it, and synchronises the device while doing so.  0 = no kernel gave up.
+ */
+moepp_status moepp_device_error(int32_t* code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOEPP_H */

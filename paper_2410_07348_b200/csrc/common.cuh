@@ -1,0 +1,87 @@
+// Internal declarations shared by the kernels and the C-ABI layer of the MoE++ forward library.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "moepp.h"
+
+namespace moepp {
+
+constexpr int kMaxExperts = 64;     // N
+constexpr int kMaxTopK = 8;         // K
+constexpr int kMaxRouteRows = 128;  // N + 2 * n_const
+
+struct Dims {
+  int T, D, F;
+  int n_ffn, n_zero, n_copy, n_const, N, K;
+  int dtype, renorm, row_align, add_residual, flags;
+  long long M_cap;
+  __host__ __device__ int zero0() const { return n_ffn; }
+  __host__ __device__ int copy0() const { return n_ffn + n_zero; }
+  __host__ __device__ int const0() const { return n_ffn + n_zero + n_copy; }
+};
+
+inline size_t elem_size(int dtype) { return dtype == MOEPP_BF16 ? 2 : 4; }
+
+// ---- kernel launchers (each enqueues on `st` and returns the launch status) -------------------
+cudaError_t launch_route(const Dims& d, const void* x, const float* W_r, const float* W_g, const float* prev,
+                         const float* bias, const float* W_c, float* logits, int32_t* topk_idx, float* topk_w,
+                         int32_t* counts, int32_t* offsets, float* alpha, cudaStream_t st);
+
+cudaError_t launch_permute(const Dims& d, const void* x, const int32_t* topk_idx, const int32_t* offsets,
+                           int32_t* row_of_slot, int32_t* slot_of_row, void* x_perm, cudaStream_t st);
+
+cudaError_t launch_ffn_simt(const Dims& d, const void* x_perm, const int32_t* offsets, const void* W_gate,
+                            const void* W_up, const void* W_down, void* h, void* y_perm, cudaStream_t st);
+
+// bf16 tensor-core path; returns cudaErrorNotSupported if the tensor maps cannot be encoded.
+cudaError_t launch_ffn_tcgen05(const Dims& d, const void* x_perm, const int32_t* offsets, const void* W_gate,
+                               const void* W_up, const void* W_down, void* h, void* y_perm, cudaStream_t st);
+
+cudaError_t launch_combine(const Dims& d, const void* x, const void* y_perm, const int32_t* topk_idx,
+                           const float* topk_w, const int32_t* row_of_slot, const float* alpha, const float* W_c,
+                           const float* v, void* y, cudaStream_t st);
+
+// Error word written by kernels whose bounded waits ran out (0 = fine).
+cudaError_t read_and_clear_device_error(int32_t* code);
+
+// ---- small device helpers -----------------------------------------------------------------------
+__device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&p);
+}
+
+// 8 consecutive elements of a row as floats (16 bytes of bf16, or 32 bytes of float).
+template <typename T>
+struct Vec8;
+template <>
+struct Vec8<__nv_bfloat16> {
+  static __device__ __forceinline__ void load(const __nv_bfloat16* p, float (&f)[8]) {
+    const uint4 u = *reinterpret_cast<const uint4*>(p);
+    f[0] = bf16_lo(u.x); f[1] = bf16_hi(u.x); f[2] = bf16_lo(u.y); f[3] = bf16_hi(u.y);
+    f[4] = bf16_lo(u.z); f[5] = bf16_hi(u.z); f[6] = bf16_lo(u.w); f[7] = bf16_hi(u.w);
+  }
+  static __device__ __forceinline__ void store(__nv_bfloat16* p, const float (&f)[8]) {
+    uint4 u;
+    u.x = pack_bf16(f[0], f[1]); u.y = pack_bf16(f[2], f[3]); u.z = pack_bf16(f[4], f[5]); u.w = pack_bf16(f[6], f[7]);
+    *reinterpret_cast<uint4*>(p) = u;
+  }
+};
+template <>
+struct Vec8<float> {
+  static __device__ __forceinline__ void load(const float* p, float (&f)[8]) {
+    const float4 a = *reinterpret_cast<const float4*>(p);
+    const float4 b = *reinterpret_cast<const float4*>(p + 4);
+    f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
+  }
+  static __device__ __forceinline__ void store(float* p, const float (&f)[8]) {
+    *reinterpret_cast<float4*>(p) = make_float4(f[0], f[1], f[2], f[3]);
+    *reinterpret_cast<float4*>(p + 4) = make_float4(f[4], f[5], f[6], f[7]);
+  }
+};
+
+}  // namespace moepp

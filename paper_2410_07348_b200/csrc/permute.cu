@@ -1,0 +1,117 @@
+// Grouping of the FFN slots (zero-computation slots never get a row) and the row gather.
+//   rank kernel  : stable rank of every FFN slot inside its expert -> row_of_slot, slot_of_row
+//   gather kernel: x_perm[row] = x[slot / K], 16-byte vectors, one warp per row
+// The rank is deterministic (ascending slot id inside an expert): no atomics decide placement.
+#include "common.cuh"
+
+namespace moepp {
+namespace {
+
+constexpr int kRankThreads = 1024;
+constexpr int kRankWarps = kRankThreads / 32;
+
+// One CTA.  Warp w owns a contiguous range of slots.  Pass 1 counts its slots per expert, a scan over
+// (expert, warp) turns the counts into first rows, pass 2 hands out rows in slot order.
+__global__ void __launch_bounds__(kRankThreads)
+permute_rank_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ offsets, long long S, int n_ffn,
+                    int32_t* __restrict__ row_of_slot, int32_t* __restrict__ slot_of_row) {
+  __shared__ int base[kRankWarps][kMaxExperts];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  for (int i = tid; i < kRankWarps * kMaxExperts; i += kRankThreads) (&base[0][0])[i] = 0;
+  __syncthreads();
+
+  long long per_warp = (S + kRankWarps - 1) / kRankWarps;
+  per_warp = (per_warp + 31) / 32 * 32;
+  const long long s_begin = (long long)warp * per_warp;
+  const long long s_end = (s_begin + per_warp < S) ? s_begin + per_warp : S;
+  const unsigned lt_mask = (1u << lane) - 1u;
+
+  for (long long s0 = s_begin; s0 < s_end; s0 += 32) {
+    const long long s = s0 + lane;
+    int e = (s < s_end) ? topk_idx[s] : -1;
+    if (e >= n_ffn) e = -1;
+    const unsigned peers = __match_any_sync(0xffffffffu, e);
+    if (e >= 0 && (peers & lt_mask) == 0) base[warp][e] += __popc(peers);
+    __syncwarp();
+  }
+  __syncthreads();
+  if (tid < n_ffn) {
+    int run = offsets[tid];
+    for (int w = 0; w < kRankWarps; ++w) {
+      const int c = base[w][tid];
+      base[w][tid] = run;
+      run += c;
+    }
+  }
+  __syncthreads();
+  for (long long s0 = s_begin; s0 < s_end; s0 += 32) {
+    const long long s = s0 + lane;
+    const bool live = s < s_end;
+    int e = live ? topk_idx[s] : -1;
+    if (e >= n_ffn) e = -1;
+    const unsigned peers = __match_any_sync(0xffffffffu, e);
+    int row = -1;
+    if (e >= 0) row = base[warp][e] + __popc(peers & lt_mask);
+    __syncwarp();
+    if (e >= 0 && (peers & lt_mask) == 0) base[warp][e] += __popc(peers);
+    __syncwarp();
+    if (live) {
+      row_of_slot[s] = row;
+      if (row >= 0) slot_of_row[row] = (int32_t)s;
+    }
+  }
+}
+
+// One warp per grouped row.  Rows at or beyond offsets[n_ffn] are not touched.
+template <typename XT>
+__global__ void __launch_bounds__(256)
+permute_gather_kernel(const XT* __restrict__ x, const int32_t* __restrict__ slot_of_row,
+                      const int32_t* __restrict__ offsets, int n_ffn, int K, int D, long long M_cap,
+                      XT* __restrict__ x_perm) {
+  const int lane = threadIdx.x & 31;
+  const long long row = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= M_cap) return;
+  if (row >= __ldg(offsets + n_ffn)) return;
+  const int slot = slot_of_row[row];
+  constexpr int V = 16 / sizeof(XT);  // elements per 16-byte vector
+  const int nvec = D / V;
+  uint4* dst = reinterpret_cast<uint4*>(x_perm + (size_t)row * D);
+  if (slot < 0) {
+    for (int i = lane; i < nvec; i += 32) dst[i] = make_uint4(0u, 0u, 0u, 0u);
+    return;
+  }
+  const uint4* src = reinterpret_cast<const uint4*>(x + (size_t)(slot / K) * D);
+  int i = lane;
+  for (; i + 96 < nvec; i += 128) {  // four loads in flight per lane
+    const uint4 a = __ldg(src + i), b = __ldg(src + i + 32), c = __ldg(src + i + 64), e = __ldg(src + i + 96);
+    dst[i] = a; dst[i + 32] = b; dst[i + 64] = c; dst[i + 96] = e;
+  }
+  for (; i < nvec; i += 32) dst[i] = __ldg(src + i);
+}
+
+}  // namespace
+
+cudaError_t launch_permute(const Dims& d, const void* x, const int32_t* topk_idx, const int32_t* offsets,
+                           int32_t* row_of_slot, int32_t* slot_of_row, void* x_perm, cudaStream_t st) {
+  if (d.M_cap > 0) {
+    cudaError_t err = cudaMemsetAsync(slot_of_row, 0xff, sizeof(int32_t) * (size_t)d.M_cap, st);
+    if (err != cudaSuccess) return err;
+  }
+  if (d.T == 0) return cudaSuccess;
+  const long long S = (long long)d.T * d.K;
+  permute_rank_kernel<<<1, kRankThreads, 0, st>>>(topk_idx, offsets, S, d.n_ffn, row_of_slot, slot_of_row);
+  cudaError_t err = cudaGetLastError();
+  if (err != cudaSuccess || d.n_ffn == 0 || d.M_cap == 0) return err;
+  const int rows_per_block = 8;
+  const unsigned grid = (unsigned)((d.M_cap + rows_per_block - 1) / rows_per_block);
+  if (d.dtype == MOEPP_BF16)
+    permute_gather_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(x), slot_of_row,
+                                                               offsets, d.n_ffn, d.K, d.D, d.M_cap,
+                                                               static_cast<__nv_bfloat16*>(x_perm));
+  else
+    permute_gather_kernel<float><<<grid, 256, 0, st>>>(static_cast<const float*>(x), slot_of_row, offsets, d.n_ffn,
+                                                       d.K, d.D, d.M_cap, static_cast<float*>(x_perm));
+  return cudaGetLastError();
+}
+
+}  // namespace moepp
