@@ -1,0 +1,294 @@
+// C-ABI layer: argument validation on the host, workspace carving, and the five calls of the layer.
+// Nothing here allocates memory or synchronises the stream.
+#include <cstring>
+
+#include "common.cuh"
+
+using namespace moepp;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Checks the configuration and fills the internal dimension record.
+moepp_status make_dims(const moepp_config* c, Dims* d) {
+  if (c == nullptr) return MOEPP_ERR_INVALID_ARG;
+  if (c->T < 0 || c->D <= 0 || c->F < 0) return MOEPP_ERR_INVALID_ARG;
+  if (c->n_ffn < 0 || c->n_zero < 0 || c->n_copy < 0 || c->n_const < 0) return MOEPP_ERR_INVALID_ARG;
+  const long long N = (long long)c->n_ffn + c->n_zero + c->n_copy + c->n_const;
+  if (N <= 0) return MOEPP_ERR_INVALID_ARG;
+  if (N > kMaxExperts || N + 2 * c->n_const > kMaxRouteRows) return MOEPP_ERR_UNSUPPORTED;
+  if (c->top_k < 1 || c->top_k > N) return MOEPP_ERR_INVALID_ARG;
+  if (c->top_k > kMaxTopK) return MOEPP_ERR_UNSUPPORTED;
+  if (c->dtype != MOEPP_F32 && c->dtype != MOEPP_BF16) return MOEPP_ERR_INVALID_ARG;
+  if (c->row_align < 1 || c->row_align > 4096) return MOEPP_ERR_INVALID_ARG;
+  if (c->n_ffn > 0 && c->F <= 0) return MOEPP_ERR_INVALID_ARG;
+  if (c->D % 8 != 0 || c->F % 8 != 0) return MOEPP_ERR_ALIGN;
+  const long long S = (long long)c->T * c->top_k;
+  const long long M_cap = S + (long long)c->n_ffn * (c->row_align - 1);
+  if (M_cap > 0x7fffffffLL) return MOEPP_ERR_UNSUPPORTED;  // rows and slots are int32
+  d->T = c->T; d->D = c->D; d->F = c->F;
+  d->n_ffn = c->n_ffn; d->n_zero = c->n_zero; d->n_copy = c->n_copy; d->n_const = c->n_const;
+  d->N = (int)N; d->K = c->top_k;
+  d->dtype = c->dtype; d->renorm = c->renorm_topk ? 1 : 0; d->row_align = c->row_align;
+  d->add_residual = c->add_residual ? 1 : 0; d->flags = c->flags;
+  d->M_cap = M_cap;
+  return MOEPP_OK;
+}
+
+inline moepp_status from_cuda(cudaError_t e) { return e == cudaSuccess ? MOEPP_OK : MOEPP_ERR_CUDA; }
+
+// Regions of the layer workspace, in order.  `host_io` adds device staging for x, prev, y.
+struct Carve {
+  size_t logits, topk_idx, topk_w, counts, offsets, alpha, row_of_slot, slot_of_row, x_perm, h, y_perm;
+  size_t x_dev, prev_dev, y_dev;
+  size_t total;
+};
+
+Carve carve(const Dims& d, bool host_io) {
+  Carve c{};
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    const size_t at = off;
+    off += align_up(bytes > 0 ? bytes : 1);
+    return at;
+  };
+  const size_t es = elem_size(d.dtype);
+  const size_t S = (size_t)d.T * d.K;
+  c.logits = take(sizeof(float) * (size_t)d.T * d.N);
+  c.topk_idx = take(sizeof(int32_t) * S);
+  c.topk_w = take(sizeof(float) * S);
+  c.counts = take(sizeof(int32_t) * d.N);
+  c.offsets = take(sizeof(int32_t) * (d.n_ffn + 1));
+  c.alpha = take(sizeof(float) * (size_t)d.T * d.n_const * 2);
+  c.row_of_slot = take(sizeof(int32_t) * S);
+  c.slot_of_row = take(sizeof(int32_t) * (size_t)d.M_cap);
+  c.x_perm = take(es * (size_t)d.M_cap * d.D);
+  c.h = take(es * (size_t)d.M_cap * d.F);
+  c.y_perm = take(es * (size_t)d.M_cap * d.D);
+  if (host_io) {
+    c.x_dev = take(es * (size_t)d.T * d.D);
+    c.prev_dev = take(sizeof(float) * (size_t)d.T * d.N);
+    c.y_dev = take(es * (size_t)d.T * d.D);
+  }
+  c.total = off;
+  return c;
+}
+
+moepp_status ffn_dispatch(const Dims& d, const void* x_perm, const int32_t* offsets, const void* W_gate,
+                          const void* W_up, const void* W_down, void* h, void* y_perm, cudaStream_t st) {
+  if (d.n_ffn == 0 || d.T == 0) return MOEPP_OK;
+  if (d.dtype == MOEPP_BF16 && !(d.flags & MOEPP_FLAG_SIMT_FFN)) {
+    const cudaError_t e = launch_ffn_tcgen05(d, x_perm, offsets, W_gate, W_up, W_down, h, y_perm, st);
+    if (e == cudaErrorNotSupported) return MOEPP_ERR_UNSUPPORTED;
+    return from_cuda(e);
+  }
+  return from_cuda(launch_ffn_simt(d, x_perm, offsets, W_gate, W_up, W_down, h, y_perm, st));
+}
+
+moepp_status layer_on_device(const Dims& d, const Carve& c, const moepp_weights* w, const void* x,
+                             const float* prev, void* y, float* logits_out, char* ws, cudaStream_t st) {
+  float* logits = logits_out ? logits_out : reinterpret_cast<float*>(ws + c.logits);
+  int32_t* topk_idx = reinterpret_cast<int32_t*>(ws + c.topk_idx);
+  float* topk_w = reinterpret_cast<float*>(ws + c.topk_w);
+  int32_t* counts = reinterpret_cast<int32_t*>(ws + c.counts);
+  int32_t* offsets = reinterpret_cast<int32_t*>(ws + c.offsets);
+  float* alpha = d.n_const > 0 ? reinterpret_cast<float*>(ws + c.alpha) : nullptr;
+  int32_t* row_of_slot = reinterpret_cast<int32_t*>(ws + c.row_of_slot);
+  int32_t* slot_of_row = reinterpret_cast<int32_t*>(ws + c.slot_of_row);
+  void* x_perm = ws + c.x_perm;
+  void* h = ws + c.h;
+  void* y_perm = ws + c.y_perm;
+
+  cudaError_t e = launch_route(d, x, w->W_r, w->W_g, prev, w->router_bias, w->W_c, logits, topk_idx, topk_w, counts,
+                               offsets, alpha, st);
+  if (e != cudaSuccess) return MOEPP_ERR_CUDA;
+  e = launch_permute(d, x, topk_idx, offsets, row_of_slot, slot_of_row, x_perm, st);
+  if (e != cudaSuccess) return MOEPP_ERR_CUDA;
+  const moepp_status s = ffn_dispatch(d, x_perm, offsets, w->W_gate, w->W_up, w->W_down, h, y_perm, st);
+  if (s != MOEPP_OK) return s;
+  e = launch_combine(d, x, y_perm, topk_idx, topk_w, row_of_slot, alpha, w->W_c, w->v, y, st);
+  return from_cuda(e);
+}
+
+moepp_status check_layer_args(const Dims& d, const moepp_weights* w, const void* x, const float* prev, const void* y,
+                              const void* ws) {
+  if (w == nullptr || x == nullptr || y == nullptr || ws == nullptr) return MOEPP_ERR_INVALID_ARG;
+  if (d.flags & MOEPP_FLAG_LOGITS_GIVEN) return MOEPP_ERR_INVALID_ARG;  // a whole layer computes its own logits
+  if (w->W_r == nullptr) return MOEPP_ERR_INVALID_ARG;
+  if ((w->W_g == nullptr) != (prev == nullptr)) return MOEPP_ERR_INVALID_ARG;
+  if (d.n_const > 0 && (w->W_c == nullptr || w->v == nullptr)) return MOEPP_ERR_INVALID_ARG;
+  if (d.n_ffn > 0 && (w->W_gate == nullptr || w->W_up == nullptr || w->W_down == nullptr))
+    return MOEPP_ERR_INVALID_ARG;
+  if (!aligned16(w->W_r) || !aligned16(w->W_c) || !aligned16(w->v) || !aligned16(w->W_gate) ||
+      !aligned16(w->W_up) || !aligned16(w->W_down))
+    return MOEPP_ERR_ALIGN;
+  if ((reinterpret_cast<uintptr_t>(ws) & (kAlign - 1)) != 0) return MOEPP_ERR_ALIGN;
+  return MOEPP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* moepp_status_string(moepp_status s) {
+  switch (s) {
+    case MOEPP_OK: return "ok";
+    case MOEPP_ERR_INVALID_ARG: return "invalid argument";
+    case MOEPP_ERR_UNSUPPORTED: return "unsupported configuration";
+    case MOEPP_ERR_ALIGN: return "pointer or dimension not aligned";
+    case MOEPP_ERR_WORKSPACE: return "workspace too small";
+    case MOEPP_ERR_CUDA: return "CUDA error at launch";
+    case MOEPP_ERR_TIMEOUT: return "a device-side wait ran out";
+  }
+  return "unknown status";
+}
+
+moepp_status moepp_workspace_bytes(const moepp_config* cfg, size_t* bytes) {
+  Dims d;
+  const moepp_status s = make_dims(cfg, &d);
+  if (s != MOEPP_OK) return s;
+  if (bytes == nullptr) return MOEPP_ERR_INVALID_ARG;
+  *bytes = carve(d, false).total;
+  return MOEPP_OK;
+}
+
+moepp_status moepp_workspace_bytes_host(const moepp_config* cfg, size_t* bytes) {
+  Dims d;
+  const moepp_status s = make_dims(cfg, &d);
+  if (s != MOEPP_OK) return s;
+  if (bytes == nullptr) return MOEPP_ERR_INVALID_ARG;
+  *bytes = carve(d, true).total;
+  return MOEPP_OK;
+}
+
+moepp_status moepp_route(const moepp_config* cfg, const void* x, const float* W_r, const float* W_g,
+                         const float* prev_logits, const float* router_bias, const float* W_c, float* logits,
+                         int32_t* topk_idx, float* topk_w, int32_t* expert_counts, int32_t* expert_offsets,
+                         float* alpha, void* stream) {
+  Dims d;
+  const moepp_status s = make_dims(cfg, &d);
+  if (s != MOEPP_OK) return s;
+  if (logits == nullptr || topk_idx == nullptr || topk_w == nullptr || expert_counts == nullptr ||
+      expert_offsets == nullptr)
+    return MOEPP_ERR_INVALID_ARG;
+  const bool given = (d.flags & MOEPP_FLAG_LOGITS_GIVEN) != 0;
+  if (given) {
+    W_r = nullptr; W_g = nullptr; prev_logits = nullptr; router_bias = nullptr;
+  } else {
+    if (W_r == nullptr) return MOEPP_ERR_INVALID_ARG;
+    if ((W_g == nullptr) != (prev_logits == nullptr)) return MOEPP_ERR_INVALID_ARG;
+  }
+  if (d.n_const == 0) alpha = nullptr;
+  if (alpha != nullptr && W_c == nullptr) return MOEPP_ERR_INVALID_ARG;
+  const bool needs_x = !given || alpha != nullptr;
+  if (needs_x && x == nullptr) return MOEPP_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(W_r) || !aligned16(W_c)) return MOEPP_ERR_ALIGN;
+  return from_cuda(launch_route(d, x, W_r, W_g, prev_logits, router_bias, W_c, logits, topk_idx, topk_w,
+                                expert_counts, expert_offsets, alpha, static_cast<cudaStream_t>(stream)));
+}
+
+moepp_status moepp_permute(const moepp_config* cfg, const void* x, const int32_t* topk_idx,
+                           const int32_t* expert_offsets, int32_t* row_of_slot, int32_t* slot_of_row, void* x_perm,
+                           void* stream) {
+  Dims d;
+  const moepp_status s = make_dims(cfg, &d);
+  if (s != MOEPP_OK) return s;
+  if (x == nullptr || topk_idx == nullptr || expert_offsets == nullptr || row_of_slot == nullptr ||
+      slot_of_row == nullptr || x_perm == nullptr)
+    return MOEPP_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(x_perm)) return MOEPP_ERR_ALIGN;
+  return from_cuda(launch_permute(d, x, topk_idx, expert_offsets, row_of_slot, slot_of_row, x_perm,
+                                  static_cast<cudaStream_t>(stream)));
+}
+
+moepp_status moepp_grouped_ffn(const moepp_config* cfg, const void* x_perm, const int32_t* expert_offsets,
+                               const void* W_gate, const void* W_up, const void* W_down, void* h_ws, void* y_perm,
+                               void* stream) {
+  Dims d;
+  const moepp_status s = make_dims(cfg, &d);
+  if (s != MOEPP_OK) return s;
+  if (x_perm == nullptr || expert_offsets == nullptr || h_ws == nullptr || y_perm == nullptr)
+    return MOEPP_ERR_INVALID_ARG;
+  if (d.n_ffn > 0 && (W_gate == nullptr || W_up == nullptr || W_down == nullptr)) return MOEPP_ERR_INVALID_ARG;
+  if (!aligned16(x_perm) || !aligned16(W_gate) || !aligned16(W_up) || !aligned16(W_down) || !aligned16(h_ws) ||
+      !aligned16(y_perm))
+    return MOEPP_ERR_ALIGN;
+  return ffn_dispatch(d, x_perm, expert_offsets, W_gate, W_up, W_down, h_ws, y_perm,
+                      static_cast<cudaStream_t>(stream));
+}
+
+moepp_status moepp_combine(const moepp_config* cfg, const void* x, const void* y_perm, const int32_t* topk_idx,
+                           const float* topk_w, const int32_t* row_of_slot, const float* alpha, const float* W_c,
+                           const float* v, void* y, void* stream) {
+  Dims d;
+  const moepp_status s = make_dims(cfg, &d);
+  if (s != MOEPP_OK) return s;
+  if (x == nullptr || topk_idx == nullptr || topk_w == nullptr || row_of_slot == nullptr || y == nullptr)
+    return MOEPP_ERR_INVALID_ARG;
+  if (d.n_ffn > 0 && y_perm == nullptr) return MOEPP_ERR_INVALID_ARG;
+  if (d.n_const > 0 && (v == nullptr || (alpha == nullptr && W_c == nullptr))) return MOEPP_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(y_perm) || !aligned16(y) || !aligned16(v) || !aligned16(W_c))
+    return MOEPP_ERR_ALIGN;
+  return from_cuda(launch_combine(d, x, y_perm, topk_idx, topk_w, row_of_slot, alpha, W_c, v, y,
+                                  static_cast<cudaStream_t>(stream)));
+}
+
+moepp_status moepp_layer_forward(const moepp_config* cfg, const moepp_weights* weights, const void* x,
+                                 const float* prev_logits, void* y, float* logits_out, void* workspace,
+                                 size_t workspace_bytes, void* stream) {
+  Dims d;
+  moepp_status s = make_dims(cfg, &d);
+  if (s != MOEPP_OK) return s;
+  s = check_layer_args(d, weights, x, prev_logits, y, workspace);
+  if (s != MOEPP_OK) return s;
+  if (!aligned16(x) || !aligned16(y)) return MOEPP_ERR_ALIGN;
+  const Carve c = carve(d, false);
+  if (workspace_bytes < c.total) return MOEPP_ERR_WORKSPACE;
+  return layer_on_device(d, c, weights, x, prev_logits, y, logits_out, static_cast<char*>(workspace),
+                         static_cast<cudaStream_t>(stream));
+}
+
+moepp_status moepp_layer_forward_host(const moepp_config* cfg, const moepp_weights* weights, const void* x_host,
+                                      const float* prev_logits_host, void* y_host, float* logits_out_host,
+                                      void* workspace, size_t workspace_bytes, void* stream) {
+  Dims d;
+  moepp_status s = make_dims(cfg, &d);
+  if (s != MOEPP_OK) return s;
+  s = check_layer_args(d, weights, x_host, prev_logits_host, y_host, workspace);
+  if (s != MOEPP_OK) return s;
+  const Carve c = carve(d, true);
+  if (workspace_bytes < c.total) return MOEPP_ERR_WORKSPACE;
+  if (d.T == 0) return MOEPP_OK;
+  char* ws = static_cast<char*>(workspace);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t es = elem_size(d.dtype);
+  const size_t act_bytes = es * (size_t)d.T * d.D, lg_bytes = sizeof(float) * (size_t)d.T * d.N;
+  if (cudaMemcpyAsync(ws + c.x_dev, x_host, act_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return MOEPP_ERR_CUDA;
+  const float* prev_dev = nullptr;
+  if (prev_logits_host != nullptr) {
+    if (cudaMemcpyAsync(ws + c.prev_dev, prev_logits_host, lg_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+      return MOEPP_ERR_CUDA;
+    prev_dev = reinterpret_cast<const float*>(ws + c.prev_dev);
+  }
+  s = layer_on_device(d, c, weights, ws + c.x_dev, prev_dev, ws + c.y_dev, nullptr, ws, st);
+  if (s != MOEPP_OK) return s;
+  if (cudaMemcpyAsync(y_host, ws + c.y_dev, act_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return MOEPP_ERR_CUDA;
+  if (logits_out_host != nullptr &&
+      cudaMemcpyAsync(logits_out_host, ws + c.logits, lg_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return MOEPP_ERR_CUDA;
+  return MOEPP_OK;
+}
+
+moepp_status moepp_device_error(int32_t* code) {
+  if (code == nullptr) return MOEPP_ERR_INVALID_ARG;
+  const cudaError_t e = read_and_clear_device_error(code);
+  if (e != cudaSuccess) return MOEPP_ERR_CUDA;
+  return *code == 0 ? MOEPP_OK : MOEPP_ERR_TIMEOUT;
+}
+
+}  // extern "C"

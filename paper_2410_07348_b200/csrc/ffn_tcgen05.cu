@@ -1,0 +1,419 @@
+// Grouped SwiGLU FFN of the MoE++ layer on the 5th-generation tensor cores (sm_100a), bf16 in,
+// float accumulation in tensor memory.  Two launches of one persistent, warp-specialised kernel:
+//   GEMM 1  h[r,:]      = silu(x_perm[r,:] W_gate[e]^T) * (x_perm[r,:] W_up[e]^T)   (SwiGLU epilogue)
+//   GEMM 2  y_perm[r,:] = h[r,:] W_down[e]^T
+// for every FFN expert e and every row r of its segment [offsets[e], offsets[e+1]).
+//
+// Per CTA (one per SM): warp 0 = TMA producer, warp 1 = MMA issuer (tcgen05.mma, one thread),
+// warps 2-5 = epilogue (tcgen05.ld -> registers -> global).  Operand tiles (128 rows x 64 k of A,
+// 256 rows x 64 k of B, 128-byte swizzle) move through a 4-stage shared-memory ring guarded by
+// mbarriers; the 128 x 256 float accumulator is double-buffered in the 512 TMEM columns so that the
+// epilogue of one tile overlaps the MMAs of the next.  For GEMM 1 the 256 accumulator columns are
+// 128 gate columns followed by the matching 128 up columns, so SwiGLU needs no second pass.
+// The tile list depends on the routing (offsets lives on the device): every role walks the same
+// static schedule tile = blockIdx.x + i * gridDim.x and decodes it from a small table in shared memory.
+// Every wait is bounded: a wait that runs out raises an error word and the CTA drains and leaves.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace moepp {
+
+__device__ int32_t g_device_error = 0;
+
+cudaError_t read_and_clear_device_error(int32_t* code) {
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return e;
+  e = cudaMemcpyFromSymbol(code, g_device_error, sizeof(int32_t));
+  if (e != cudaSuccess) return e;
+  const int32_t zero = 0;
+  return cudaMemcpyToSymbol(g_device_error, &zero, sizeof(int32_t));
+}
+
+namespace {
+
+constexpr int BM = 128;      // rows per tile (UMMA M)
+constexpr int BK = 64;       // k elements per stage: 128 bytes of bf16 = one swizzle row
+constexpr int UMMA_N = 256;  // accumulator columns per tile
+constexpr int UMMA_K = 16;   // k per tcgen05.mma for 16-bit operands
+constexpr int kStages = 4;
+constexpr int kABytes = BM * BK * 2;          // 16 KiB
+constexpr int kBBytes = UMMA_N * BK * 2;      // 32 KiB
+constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kThreads = 192;
+constexpr int kTmemCols = 512;
+constexpr int kSmemBytes = kStages * kStageBytes + 1024;  // + slack to align the ring to 1024 B
+constexpr long long kWaitCycles = 4000000000LL;           // about two seconds: far beyond any healthy wait
+
+// instruction descriptor: D = f32, A = B = bf16, both K-major, N = 256, M = 128
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((UMMA_N >> 3) << 17) | ((BM >> 4) << 24);
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
+// Bounded wait.  Returns false if the CTA is giving up (this wait ran out, or another one did).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int code) {
+  long long t0 = 0;
+  for (uint32_t spin = 0;; ++spin) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (spin >= 1024u) {
+      if (spin == 1024u) t0 = clock64();
+      if (*abort_flag != 0) return false;
+      if (clock64() - t0 > kWaitCycles) {
+        *abort_flag = code;
+        atomicCAS(&g_device_error, 0, code);
+        return false;
+      }
+      __nanosleep(64);
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1)
+      : "memory");
+}
+
+// shared-memory matrix descriptor: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)1 << 16;             // leading byte offset (not used by swizzled K-major layouts)
+  d |= (uint64_t)(1024 >> 4) << 32;   // stride byte offset
+  d |= (uint64_t)1 << 46;             // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;             // 128-byte swizzle
+  return d;
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(kIdesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// 16 consecutive accumulator columns of this thread's TMEM lane
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// Ties the loaded registers to a point after the wait, so that no use of them is scheduled before it.
+__device__ __forceinline__ void tmem_ld_pin(uint32_t (&r)[16]) {
+  asm volatile("" : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                    "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]),
+                    "+r"(r[15])
+               :
+               : "memory");
+}
+
+__device__ __forceinline__ float silu_mul(float g, float u) { return __fdividef(g, 1.f + __expf(-g)) * u; }
+
+struct TileInfo {
+  int e, row0, row_end, n0;
+};
+
+// SWIGLU: C has Nout columns, the tile covers 128 of them (gate | up in the accumulator).
+// otherwise the tile covers 256 columns of C.
+template <bool SWIGLU>
+__global__ void __launch_bounds__(kThreads, 1)
+grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
+                    const __grid_constant__ CUtensorMap tmB1, __nv_bfloat16* __restrict__ C,
+                    const int32_t* __restrict__ offsets, int n_ffn, int Nout, int Kd) {
+  constexpr int BN_OUT = SWIGLU ? 128 : 256;
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bar_full[kStages], bar_empty[kStages], bar_tmem_full[2], bar_tmem_empty[2],
+      bar_drain;
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int tile_start[kMaxExperts + 1];
+  __shared__ int seg_begin[kMaxExperts + 1];
+  __shared__ volatile int abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const int NT = (Nout + BN_OUT - 1) / BN_OUT;
+  const int KB = (Kd + BK - 1) / BK;
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(smem_u32(&bar_full[s]), 1);
+      mbar_init(smem_u32(&bar_empty[s]), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&bar_tmem_full[b]), 1);
+      mbar_init(smem_u32(&bar_tmem_empty[b]), 4);
+    }
+    mbar_init(smem_u32(&bar_drain), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    int run = 0;
+    for (int e = 0; e < n_ffn; ++e) {
+      const int b = offsets[e], en = offsets[e + 1];
+      seg_begin[e] = b;
+      tile_start[e] = run;
+      run += ((en - b + BM - 1) / BM) * NT;
+    }
+    seg_begin[n_ffn] = offsets[n_ffn];
+    tile_start[n_ffn] = run;
+  }
+  if (warp == 1) {  // TMEM: all 512 columns (two accumulators)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
+                 "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+  const int total_tiles = tile_start[n_ffn];
+
+  // decode a linear tile index; `e` only moves forward
+  auto decode = [&](int L, int& e) -> TileInfo {
+    while (L >= tile_start[e + 1]) ++e;
+    const int local = L - tile_start[e];
+    const int b = seg_begin[e], en = seg_begin[e + 1];
+    const int mt = (en - b + BM - 1) / BM;
+    TileInfo ti;
+    ti.e = e;
+    ti.row0 = b + (local % mt) * BM;
+    ti.row_end = en;
+    ti.n0 = (local / mt) * BN_OUT;
+    return ti;
+  };
+
+  if (warp == 0) {
+    // ---------------------------------- TMA producer ---------------------------------------------
+    if (lane == 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB0) : "memory");
+      if (SWIGLU) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB1) : "memory");
+      uint32_t it = 0;
+      int e = 0;
+      bool ok = true;
+      for (int L = blockIdx.x; L < total_tiles && ok; L += gridDim.x) {
+        const TileInfo ti = decode(L, e);
+        const int brow = ti.e * Nout + ti.n0;
+        for (int kb = 0; kb < KB; ++kb, ++it) {
+          const uint32_t s = it % kStages, ph = (it / kStages) & 1u;
+          if (!mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u, &abort_flag, 1)) { ok = false; break; }
+          const uint32_t full = smem_u32(&bar_full[s]);
+          const uint32_t a_dst = ring + s * kStageBytes, b_dst = a_dst + kABytes;
+          mbar_expect_tx(full, kStageBytes);
+          tma_load_2d(a_dst, &tmA, kb * BK, ti.row0, full);
+          if (SWIGLU) {
+            tma_load_2d(b_dst, &tmB0, kb * BK, brow, full);
+            tma_load_2d(b_dst + kBBytes / 2, &tmB1, kb * BK, brow, full);
+          } else {
+            tma_load_2d(b_dst, &tmB0, kb * BK, brow, full);
+          }
+        }
+      }
+      if (!ok) {  // give the copies already issued a bounded chance to land before the CTA leaves
+        const uint32_t n_back = it < (uint32_t)kStages ? it : (uint32_t)kStages;
+        for (uint32_t i = 1; i <= n_back; ++i) {
+          const uint32_t j = it - i, s = j % kStages, ph = (j / kStages) & 1u;
+          for (int spin = 0; spin < 100000 && !mbar_try_wait(smem_u32(&bar_full[s]), ph); ++spin) __nanosleep(64);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------- MMA issuer -----------------------------------------------
+    if (lane == 0) {
+      uint32_t it = 0, tile_iter = 0;
+      bool ok = true;
+      for (int L = blockIdx.x; L < total_tiles && ok; L += gridDim.x, ++tile_iter) {
+        const uint32_t buf = tile_iter & 1u, tph = (tile_iter >> 1) & 1u;
+        if (!mbar_wait(smem_u32(&bar_tmem_empty[buf]), tph ^ 1u, &abort_flag, 2)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * UMMA_N;
+        for (int kb = 0; kb < KB; ++kb, ++it) {
+          const uint32_t s = it % kStages, ph = (it / kStages) & 1u;
+          if (!mbar_wait(smem_u32(&bar_full[s]), ph, &abort_flag, 3)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_addr = ring + s * kStageBytes, b_addr = a_addr + kABytes;
+          const uint64_t adesc = make_smem_desc(a_addr), bdesc = make_smem_desc(b_addr);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            // advancing k by 16 elements = 32 bytes inside the 128-byte swizzle row: +2 in the address field
+            umma_bf16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), (kb | k) != 0 ? 1u : 0u);
+          }
+          umma_commit(smem_u32(&bar_empty[s]));  // stage reusable once these MMAs have read it
+        }
+        if (ok) umma_commit(smem_u32(&bar_tmem_full[buf]));  // accumulator complete
+      }
+      if (!ok) {  // let issued MMAs retire (bounded) before TMEM is released
+        umma_commit(smem_u32(&bar_drain));
+        for (int spin = 0; spin < 100000 && !mbar_try_wait(smem_u32(&bar_drain), 0); ++spin) __nanosleep(64);
+      }
+    }
+  } else {
+    // ---------------------------------- epilogue: 4 warps, one TMEM lane quarter each --------------
+    const int q = warp & 3;  // lanes [32q, 32q+32) are the ones this warp may read
+    uint32_t tile_iter = 0;
+    int e = 0;
+    bool ok = true;
+    for (int L = blockIdx.x; L < total_tiles && ok; L += gridDim.x, ++tile_iter) {
+      const TileInfo ti = decode(L, e);
+      const uint32_t buf = tile_iter & 1u, tph = (tile_iter >> 1) & 1u;
+      if (!mbar_wait(smem_u32(&bar_tmem_full[buf]), tph, &abort_flag, 4)) { ok = false; break; }
+      tc_fence_after();
+      const int grow = ti.row0 + q * 32 + lane;
+      const bool row_ok = grow < ti.row_end;
+      const uint32_t t_row = tmem_base + buf * UMMA_N + ((uint32_t)(q * 32) << 16);
+      __nv_bfloat16* crow = C + (size_t)grow * Nout + ti.n0;
+      if (SWIGLU) {
+#pragma unroll 1
+        for (int c = 0; c < 128; c += 16) {
+          uint32_t g[16], u[16];
+          tmem_ld16(t_row + c, g);
+          tmem_ld16(t_row + 128 + c, u);
+          tmem_ld_wait();
+          tmem_ld_pin(g);
+          tmem_ld_pin(u);
+          uint32_t o[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            o[i] = pack_bf16(silu_mul(__uint_as_float(g[2 * i]), __uint_as_float(u[2 * i])),
+                             silu_mul(__uint_as_float(g[2 * i + 1]), __uint_as_float(u[2 * i + 1])));
+          if (row_ok) {
+            if (ti.n0 + c + 8 <= Nout) *reinterpret_cast<uint4*>(crow + c) = make_uint4(o[0], o[1], o[2], o[3]);
+            if (ti.n0 + c + 16 <= Nout) *reinterpret_cast<uint4*>(crow + c + 8) = make_uint4(o[4], o[5], o[6], o[7]);
+          }
+        }
+      } else {
+#pragma unroll 1
+        for (int c = 0; c < 256; c += 32) {
+          uint32_t a[16], b[16];
+          tmem_ld16(t_row + c, a);
+          tmem_ld16(t_row + c + 16, b);
+          tmem_ld_wait();
+          tmem_ld_pin(a);
+          tmem_ld_pin(b);
+          uint32_t o[16];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            o[i] = pack_bf16(__uint_as_float(a[2 * i]), __uint_as_float(a[2 * i + 1]));
+            o[8 + i] = pack_bf16(__uint_as_float(b[2 * i]), __uint_as_float(b[2 * i + 1]));
+          }
+          if (row_ok) {
+#pragma unroll
+            for (int v = 0; v < 4; ++v)
+              if (ti.n0 + c + 8 * v + 8 <= Nout)
+                *reinterpret_cast<uint4*>(crow + c + 8 * v) = make_uint4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bar_tmem_empty[buf]));
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+// ---- host side: tensor maps ---------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn == nullptr) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// [rows, cols] bf16 row-major matrix, box = box_rows x 64 columns, 128-byte swizzle, zero fill outside
+bool make_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr || rows == 0) return false;
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {cols * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)BK, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+cudaError_t launch_ffn_tcgen05(const Dims& d, const void* x_perm, const int32_t* offsets, const void* W_gate,
+                               const void* W_up, const void* W_down, void* h, void* y_perm, cudaStream_t st) {
+  if (d.T == 0 || d.n_ffn == 0 || d.M_cap == 0) return cudaSuccess;
+  int dev = 0, sms = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return err;
+  err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (err != cudaSuccess) return err;
+
+  CUtensorMap mA1, mG, mU, mA2, mD;
+  const uint64_t rows = (uint64_t)d.M_cap;
+  if (!make_map(&mA1, x_perm, rows, (uint64_t)d.D, BM) ||
+      !make_map(&mG, W_gate, (uint64_t)d.n_ffn * d.F, (uint64_t)d.D, 128) ||
+      !make_map(&mU, W_up, (uint64_t)d.n_ffn * d.F, (uint64_t)d.D, 128) ||
+      !make_map(&mA2, h, rows, (uint64_t)d.F, BM) ||
+      !make_map(&mD, W_down, (uint64_t)d.n_ffn * d.D, (uint64_t)d.F, 256))
+    return cudaErrorNotSupported;
+
+  auto k1 = grouped_gemm_kernel<true>;
+  auto k2 = grouped_gemm_kernel<false>;
+  err = cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  if (err != cudaSuccess) return err;
+  err = cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  if (err != cudaSuccess) return err;
+
+  k1<<<sms, kThreads, kSmemBytes, st>>>(mA1, mG, mU, static_cast<__nv_bfloat16*>(h), offsets, d.n_ffn, d.F, d.D);
+  err = cudaGetLastError();
+  if (err != cudaSuccess) return err;
+  k2<<<sms, kThreads, kSmemBytes, st>>>(mA2, mD, mD, static_cast<__nv_bfloat16*>(y_perm), offsets, d.n_ffn, d.D, d.F);
+  return cudaGetLastError();
+}
+
+}  // namespace moepp

@@ -1,0 +1,224 @@
+"""Whole-layer GPU parity against the CPU oracle on the benchmark configurations, through the C-ABI.
+
+For every configuration: logits within 1e-4 of the oracle, top-K picks bit-exact on every token whose
+leading logits are more than 1e-3 apart, and the layer output compared with the oracle run on the
+GPU's own picks (so that every token's arithmetic is checked even where a near-tie went the other way):
+float32 within max-abs 1e-4, bf16 within per-token relative error 2e-2.  Large configurations are
+checked on a token sample (tokens are independent through the layer and through a stack).
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from harness import clear_gap_tokens, f32, max_abs, oracle_inputs, rel_err_per_token, sample_tokens, shape_of
+from paper_2410_07348_b200 import binding as B
+from paper_2410_07348_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+F32_ABS_TOL = 1e-4
+BF16_REL_TOL = 2e-2
+LOGIT_TOL = 2e-4
+
+
+def gpu_layer(cfg, wd, x, prev, host=False):
+    """Runs moepp_layer_forward (or its host-buffer variant) and, with the same inputs, moepp_route to
+    expose the picks the layer used."""
+    T, N, K = cfg.T, cfg.N, cfg.top_k
+    td = torch.bfloat16 if cfg.dtype == B.MOEPP_BF16 else torch.float32
+    if host:
+        ws = torch.empty(B.moepp_workspace_bytes(cfg, host=True), dtype=torch.uint8, device="cuda")
+        xh = x.cpu().pin_memory()
+        ph = None if prev is None else prev.cpu().pin_memory()
+        yh = torch.empty(T, cfg.D, dtype=td).pin_memory()
+        lh = torch.empty(T, N).pin_memory()
+        B.moepp_layer_forward_host(cfg, wd, xh, ph, yh, lh, ws)
+        torch.cuda.synchronize()
+        y, logits = yh.cuda(), lh.cuda()
+    else:
+        ws = torch.empty(B.moepp_workspace_bytes(cfg), dtype=torch.uint8, device="cuda")
+        y = torch.empty(T, cfg.D, dtype=td, device="cuda")
+        logits = torch.empty(T, N, device="cuda")
+        B.moepp_layer_forward(cfg, wd, x, prev, y, logits, ws)
+    idx = torch.empty(T, K, dtype=torch.int32, device="cuda")
+    w = torch.empty(T, K, device="cuda")
+    counts = torch.empty(N, dtype=torch.int32, device="cuda")
+    offsets = torch.empty(cfg.n_ffn + 1, dtype=torch.int32, device="cuda")
+    lg2 = torch.empty(T, N, device="cuda")
+    B.moepp_route(cfg, x, wd["W_r"], wd["W_g"], prev, wd["router_bias"], None, lg2, idx, w, counts, offsets, None)
+    torch.cuda.synchronize()
+    assert B.moepp_device_error() == 0
+    assert torch.equal(lg2, logits)
+    return y, logits, idx.cpu().numpy(), counts.cpu().numpy()
+
+
+def check_layer(oracle64, lt, n_sample, host=False, **over):
+    spec = lt.spec
+    cfg = B.config_from_spec(spec, **over)
+    wd = B.weights_from_tensors(lt)
+    x, prev = lt.x.cuda(), None if lt.prev is None else lt.prev.cuda()
+    y, logits, idx_g, counts = gpu_layer(cfg, wd, x, prev, host=host)
+    s, oi = shape_of(spec, **{k: v for k, v in over.items() if k in ("renorm_topk", "row_align", "add_residual")}), \
+        oracle_inputs(lt)
+    toks = None if n_sample is None else sample_tokens(idx_g, spec.N, n_sample)
+    r = oracle64.layer_forward(s, oi["x"], oi["W_r"], oi["W_g"], oi["prev"], oi["bias"], oi["W_c"], oi["v"],
+                               oi["W_gate"], oi["W_up"], oi["W_down"], forced_idx=idx_g, tokens=toks)
+    lg = logits.cpu().numpy()
+    assert max_abs(lg, r["logits"]) <= LOGIT_TOL
+    idx_o, _ = oracle64.gate_topk(s, r["logits"])
+    clear = clear_gap_tokens(r["logits"], spec.top_k)
+    assert np.array_equal(idx_g[clear], idx_o[clear])
+    assert clear.mean() > 0.9
+    got = y.float().cpu().numpy()
+    got = got if toks is None else got[toks]
+    if spec.dtype == "f32":
+        assert max_abs(got, r["y"]) <= F32_ABS_TOL
+    else:
+        assert rel_err_per_token(got, r["y"]) <= BF16_REL_TOL
+    assert counts.sum() == spec.T * spec.top_k
+    return dict(zc_share=float(counts[spec.n_ffn:].sum()) / max(1, counts.sum()), counts=counts)
+
+
+def test_cfg1_tiny_f32(oracle64, oracle32):
+    lt = W.make_config("cfg1_tiny_f32")
+    info = check_layer(oracle64, lt, None)
+    assert 0.2 < info["zc_share"] < 0.5
+    check_layer(oracle64, lt, None, renorm_topk=1, add_residual=1, row_align=128)
+    check_layer(oracle64, lt, None, host=True)
+
+
+def test_cfg1_vanilla_and_first_layer(oracle64):
+    lt = W.make_layer(W.CONFIGS["cfg1_tiny_f32"].vanilla(), seed=0, with_prev=False)
+    check_layer(oracle64, lt, None)
+
+
+def test_cfg2_bf16(oracle64):
+    lt = W.make_config("cfg2_bf16_8e", gen_device="cuda", device="cuda")
+    info = check_layer(oracle64, lt, 192)
+    assert 0.2 < info["zc_share"] < 0.5
+    check_layer(oracle64, lt, 64, host=True)
+    check_layer(oracle64, lt, 64, flags=B.FLAG_SIMT_FFN)
+
+
+def test_cfg3_bf16_skewed(oracle64):
+    lt = W.make_config("cfg3_bf16_16e_skew", gen_device="cuda", device="cuda")
+    info = check_layer(oracle64, lt, 96)
+    assert abs(info["zc_share"] - 0.30) < 0.02
+    c = info["counts"][:16].astype(np.float64)
+    assert c[0] > 8 * c[15]  # Zipf(1.1) over 16 experts: rank 1 carries about 21x rank 16
+
+
+def test_cfg4_stack_of_four(oracle64):
+    """Free-running 4-layer stack on all 32768 tokens; the oracle follows the same picks on a token sample."""
+    spec = W.CONFIGS["cfg4_7b_stack"]
+    n_tok = 48
+    rng = np.random.default_rng(0)
+    toks = np.sort(rng.choice(spec.T, n_tok, replace=False)).astype(np.int32)
+    sub = W.LayerSpec(n_tok, spec.D, spec.F, spec.n_ffn, spec.n_zero, spec.n_copy, spec.n_const, spec.top_k, "bf16")
+    cfg = B.config_from_spec(spec, add_residual=1)
+    ws = torch.empty(B.moepp_workspace_bytes(cfg), dtype=torch.uint8, device="cuda")
+    x = None
+    prev = None
+    x_o = None
+    prev_o = None
+    s_sub = shape_of(sub, add_residual=1)
+    for j in range(1, 5):
+        # build one layer at a time to bound memory: same recipe as workloads.make_stack
+        lt = W.make_layer(spec if j == 1 else W.LayerSpec(0, spec.D, spec.F, spec.n_ffn, dtype="bf16"), seed=j - 1,
+                          with_prev=False, w_std=0.02 / math.sqrt(j), device="cuda", gen_device="cuda")
+        if j == 1:
+            x = lt.x
+            x_o = f32(x)[toks]
+        else:
+            g = torch.Generator(device="cuda").manual_seed(1000 + j)
+            lt.W_g = W._randn(g, (spec.N, spec.N), 0.02 / math.sqrt(j), torch.float32, "cuda")
+        lt.spec = spec
+        wd = B.weights_from_tensors(lt)
+        y = torch.empty_like(x)
+        logits = torch.empty(spec.T, spec.N, device="cuda")
+        B.moepp_layer_forward(cfg, wd, x, prev, y, logits, ws)
+        idx = torch.empty(spec.T, spec.top_k, dtype=torch.int32, device="cuda")
+        wk = torch.empty(spec.T, spec.top_k, device="cuda")
+        cnt = torch.empty(spec.N, dtype=torch.int32, device="cuda")
+        off = torch.empty(spec.n_ffn + 1, dtype=torch.int32, device="cuda")
+        lg2 = torch.empty_like(logits)
+        B.moepp_route(cfg, x, wd["W_r"], wd["W_g"], prev, None, None, lg2, idx, wk, cnt, off, None)
+        torch.cuda.synchronize()
+        assert B.moepp_device_error() == 0
+        idx_g = idx.cpu().numpy()[toks]
+        # oracle on the sampled tokens, float activations carried from layer to layer
+        lt.x = None
+        lt.prev = None
+        oi = oracle_inputs(lt)
+        r = oracle64.layer_forward(s_sub, x_o, oi["W_r"], oi["W_g"], prev_o, None, oi["W_c"], oi["v"], oi["W_gate"],
+                                   oi["W_up"], oi["W_down"], forced_idx=idx_g)
+        got = y.float().cpu().numpy()[toks]
+        assert rel_err_per_token(got, r["y"]) <= BF16_REL_TOL, "layer %d" % j
+        lg = logits.cpu().numpy()[toks]
+        assert max_abs(lg, r["logits"]) <= 5e-2  # inputs differ by the bf16 rounding carried down the stack
+        idx_o, _ = oracle64.gate_topk(s_sub, r["logits"])
+        clear = clear_gap_tokens(r["logits"], spec.top_k, gap=0.1)
+        assert np.array_equal(idx_g[clear], idx_o[clear])
+        x, prev = y, logits
+        x_o, prev_o = r["y"], r["logits"]
+        del lt, wd
+
+
+def test_cfg4_teacher_forced_layers(oracle64):
+    """Each layer of the stack fed the oracle's own state (rounded once to bf16): picks exact, outputs in tolerance."""
+    spec = W.CONFIGS["cfg4_7b_stack"]
+    T = 256
+    sub = W.LayerSpec(T, spec.D, spec.F, spec.n_ffn, spec.n_zero, spec.n_copy, spec.n_const, spec.top_k, "bf16")
+    s = shape_of(sub, add_residual=1)
+    cfg = B.config_from_spec(sub, add_residual=1)
+    x_o = None
+    prev_o = None
+    for j in range(1, 5):
+        lt = W.make_layer(sub if j == 1 else W.LayerSpec(0, spec.D, spec.F, spec.n_ffn, dtype="bf16"), seed=j - 1,
+                          with_prev=False, w_std=0.02 / math.sqrt(j), device="cuda", gen_device="cuda")
+        if j == 1:
+            x_t = lt.x
+        else:
+            g = torch.Generator(device="cuda").manual_seed(1000 + j)
+            lt.W_g = W._randn(g, (spec.N, spec.N), 0.02 / math.sqrt(j), torch.float32, "cuda")
+            x_t = torch.from_numpy(x_o).to(torch.bfloat16).cuda()
+        lt.spec, lt.x = sub, x_t
+        lt.prev = None if prev_o is None else torch.from_numpy(prev_o).cuda()
+        check_layer(oracle64, lt, 32, add_residual=1)
+        oi = oracle_inputs(lt)
+        r = oracle64.layer_forward(s, oi["x"], oi["W_r"], oi["W_g"], oi["prev"], None, oi["W_c"], oi["v"], oi["W_gate"],
+                                   oi["W_up"], oi["W_down"], tokens=np.arange(T, dtype=np.int32))
+        x_o, prev_o = r["y"], r["logits"]
+
+
+@pytest.mark.parametrize("T,share", [(128, 0.0), (128, 0.5), (2048, 0.15), (2048, 0.75), (32768, 0.30)])
+def test_cfg5_sweep_points(oracle64, T, share):
+    lt = W.make_config("cfg5_sweep", T=T, zc_share=share, gen_device="cuda", device="cuda")
+    info = check_layer(oracle64, lt, 48)
+    assert abs(info["zc_share"] - share) < 0.03
+
+
+def test_empty_and_degenerate(oracle64):
+    # T = 0 is valid and does nothing
+    spec = W.LayerSpec(T=0, D=64, F=64, n_ffn=2, dtype="bf16")
+    lt = W.make_layer(spec, seed=0)
+    cfg = B.config_from_spec(spec)
+    ws = torch.empty(B.moepp_workspace_bytes(cfg), dtype=torch.uint8, device="cuda")
+    y = torch.empty(0, 64, dtype=torch.bfloat16, device="cuda")
+    B.moepp_layer_forward(cfg, B.weights_from_tensors(lt), lt.x.cuda(), lt.prev.cuda(), y, None, ws)
+    torch.cuda.synchronize()
+    # a layer of zero-computation experts only (no FFN expert at all)
+    spec = W.LayerSpec(T=100, D=64, F=0, n_ffn=0, n_zero=1, n_copy=1, n_const=2, dtype="f32")
+    check_layer(oracle64, W.make_layer(spec, seed=1), None)
+    # every slot on zero-computation experts although FFN experts exist: no FFN work at all
+    spec = W.LayerSpec(T=300, D=128, F=256, n_ffn=4, dtype="bf16")
+    lt = W.make_layer(spec, seed=2)
+    lt.bias = torch.tensor([-50.0] * 4 + [50.0] * 4)
+    info = check_layer(oracle64, lt, None)
+    assert info["zc_share"] == 1.0
+    # top-1 and top-4
+    for k in (1, 4):
+        spec = W.LayerSpec(T=200, D=128, F=256, n_ffn=6, top_k=k, dtype="bf16")
+        check_layer(oracle64, W.make_layer(spec, seed=3), None)
