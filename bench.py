@@ -1,0 +1,390 @@
+"""Benchmark of the MoE++ expert-forward path (arXiv 2410.07348) on B200.
+
+One step = one pass of the whole hot path (route -> permute -> grouped SwiGLU FFN -> combine) over one batch
+of the 7B-class configuration: 4 chained layers, T=32768 tokens, d_model=4096, d_ffn=2816, 16 FFN + 4
+zero-computation experts, top-2, bf16 storage with float router and accumulation.  The metric is
+expert-forward tokens/s, counted per layer (4*T tokens pass a layer per step).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload cfg4|cfg2|cfg3]
+
+Prints one JSON line (rank 0).  `value` is timed with inputs resident in HBM; `e2e` goes through the
+host-buffer C-ABI call with the copies inside the timed region; `roofline` is for the grouped FFN GEMM
+kernel; `vanilla` is the same library run as an all-FFN MoE of equal size; `cpu_baseline` is the CPU
+oracle timed on this machine's cores on a bounded token sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+METRIC = "moepp_expert_forward_tokens_per_s"
+UNIT = "tokens/s"
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm_gbs=d["hbm_gbs"], burst=d["bf16_tflops"], sustained=d.get("bf16_tflops_sustained",
+                                                                                  d["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, burst=1590.0, sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+                for n, v in zip(names, r[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            except (ValueError, IndexError):
+                pass
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+WORKLOADS = {  # name -> (config key, layers)
+    "cfg4": ("cfg4_7b_stack", 4),
+    "cfg3": ("cfg3_bf16_16e_skew", 1),
+    "cfg2": ("cfg2_bf16_8e", 1),
+}
+
+
+def build_stack(name, W, device):
+    """Layer tensors of the workload, generated on the device with seeded generators."""
+    key, n_layers = WORKLOADS[name]
+    spec = W.CONFIGS[key]
+    if n_layers > 1:
+        return spec, W.make_stack(spec, n_layers, device=device, gen_device=device)
+    return spec, [W.make_config(key, device=device, gen_device=device)]
+
+
+def vanilla_weights(wd, spec):
+    n = spec.n_ffn
+    out = dict(wd)
+    out["W_r"] = wd["W_r"][:n].contiguous()
+    out["W_g"] = None if wd["W_g"] is None else wd["W_g"][:n, :n].contiguous()
+    out["W_c"], out["v"] = None, None
+    out["router_bias"] = None if wd["router_bias"] is None else wd["router_bias"][:n].contiguous()
+    return out
+
+
+def run_reference(args, rank):
+    """The CPU oracle on this machine's cores, on a bounded token sample of the same workload."""
+    if rank != 0:
+        return
+    import numpy as np
+    import oracle
+    from oracle.adapters import oracle_inputs, shape_of
+    from paper_2410_07348_b200 import workloads as W
+    key, n_layers = WORKLOADS[args.workload]
+    spec = W.CONFIGS[key]
+    n_tok = args.ref_tokens
+    sub = W.LayerSpec(n_tok, spec.D, spec.F, spec.n_ffn, spec.n_zero, spec.n_copy, spec.n_const, spec.top_k, spec.dtype)
+    orc = oracle.Oracle("f32")
+    layers = W.make_stack(sub, n_layers) if n_layers > 1 else [W.make_layer(sub, seed=0)]
+    ois = [oracle_inputs(lt) for lt in layers]
+    shape = shape_of(sub, add_residual=1 if n_layers > 1 else 0)
+
+    def step():
+        x, prev = ois[0]["x"], ois[0]["prev"]
+        for oi in ois:
+            r = orc.layer_forward(shape, x, oi["W_r"], oi["W_g"], prev if oi["W_g"] is not None else None, None,
+                                  oi["W_c"], oi["v"], oi["W_gate"], oi["W_up"], oi["W_down"])
+            x, prev = r["y"], r["logits"]
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / args.steps
+    val = n_tok * n_layers / dt
+    sample = "%d tokens through %d layer(s) per step, float arithmetic" % (n_tok, n_layers)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": key, "layers": n_layers, "T": spec.T, "D": spec.D, "F": spec.F,
+                   "experts": "%d+%d" % (spec.n_ffn, spec.n_zc), "top_k": spec.top_k, "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def cpu_baseline(name, budget_s=15.0):
+    import numpy as np
+    import oracle
+    from oracle.adapters import oracle_inputs, shape_of
+    from paper_2410_07348_b200 import workloads as W
+    key, n_layers = WORKLOADS[name]
+    spec = W.CONFIGS[key]
+    orc = oracle.Oracle("f32")
+
+    def run(n_tok):
+        sub = W.LayerSpec(n_tok, spec.D, spec.F, spec.n_ffn, spec.n_zero, spec.n_copy, spec.n_const, spec.top_k,
+                          spec.dtype)
+        lt = W.make_layer(sub, seed=0, with_prev=(n_layers == 1))
+        oi = oracle_inputs(lt)
+        t0 = time.perf_counter()
+        orc.layer_forward(shape_of(sub), oi["x"], oi["W_r"], oi["W_g"], oi["prev"], None, oi["W_c"], oi["v"],
+                          oi["W_gate"], oi["W_up"], oi["W_down"])
+        return time.perf_counter() - t0
+
+    probe = 16
+    dt = run(probe)
+    n_tok = int(max(probe, min(4096, budget_s / max(dt / probe, 1e-9))))
+    dt = run(n_tok)
+    return {"value": n_tok / dt, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
+            "sample": "first layer of the workload on %d tokens (per-token cost does not depend on T), float "
+                      "arithmetic, %.1f s" % (n_tok, dt)}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="moepp", choices=["moepp", "reference"])
+    ap.add_argument("--workload", default="cfg4", choices=sorted(WORKLOADS))
+    ap.add_argument("--ref-tokens", type=int, default=64)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "moepp" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    from paper_2410_07348_b200 import binding as B
+    from paper_2410_07348_b200 import build as build_mod
+    from paper_2410_07348_b200 import workloads as W
+    from paper_2410_07348_b200.replicas import whole_job_rate
+    if rank == 0 or world == 1:
+        build_mod.build()
+    torch.cuda.set_device(local_rank)
+    dev = "cuda:%d" % local_rank
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+        dist.barrier()
+    B.lib()
+
+    peaks = load_peaks()
+    spec, layers = build_stack(args.workload, W, dev)
+    L = len(layers)
+    add_res = 1 if L > 1 else 0
+    cfg = B.config_from_spec(spec, add_residual=add_res)
+    cfg_v = B.config_from_spec(spec.vanilla(), add_residual=add_res)
+    wds = [B.weights_from_tensors(lt, dev) for lt in layers]
+    wds_v = [vanilla_weights(wd, spec) for wd in wds]
+    x0 = layers[0].x
+    prev0 = layers[0].prev
+    prev0_v = None if prev0 is None else prev0[:, :spec.n_ffn].contiguous()
+    ws = torch.empty(max(B.moepp_workspace_bytes(cfg, host=True), B.moepp_workspace_bytes(cfg_v, host=True)),
+                     dtype=torch.uint8, device=dev)
+    xs = [torch.empty_like(x0) for _ in range(2)]
+    lgs = [torch.empty(spec.T, spec.N, device=dev) for _ in range(2)]
+    lgs_v = [torch.empty(spec.T, spec.n_ffn, device=dev) for _ in range(2)]
+
+    def step(c, wlist, logit_bufs, p0):
+        x, prev = x0, p0
+        for j, wd in enumerate(wlist):
+            y, lg = xs[j & 1], logit_bufs[j & 1]
+            B.moepp_layer_forward(c, wd, x, prev if wd["W_g"] is not None else None, y, lg, ws)
+            x, prev = y, lg
+        return x
+
+    def timed(fn, steps, warmup, sampler=None):
+        for _ in range(warmup):
+            fn()
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+        if sampler:
+            sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        clocks = sampler.stop() if sampler else None
+        ms = e0.elapsed_time(e1)
+        if dist is not None:
+            dist.barrier()
+        _, ms = whole_job_rate(1.0, ms, device=dev)  # max over ranks of the device-side time
+        return ms / steps, clocks
+
+    # ---- headline: the stack with inputs resident in HBM -------------------------------------------------
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    ms_step, clocks = timed(lambda: step(cfg, wds, lgs, prev0), args.steps, args.warmup, sampler)
+    assert B.moepp_device_error() == 0
+    tokens_per_step = spec.T * L
+    value = world * tokens_per_step / (ms_step * 1e-3)
+
+    # ---- the same library as a vanilla all-FFN MoE of equal size ---------------------------------------------
+    ms_van, _ = timed(lambda: step(cfg_v, wds_v, lgs_v, prev0_v), max(3, args.steps // 2), 3)
+
+    # ---- per-call breakdown of layer 1 (staged calls, events between them) -----------------------------------
+    T, N, K = spec.T, spec.N, spec.top_k
+    td = x0.dtype
+    idx = torch.empty(T, K, dtype=torch.int32, device=dev)
+    wk = torch.empty(T, K, device=dev)
+    cnt = torch.empty(N, dtype=torch.int32, device=dev)
+    off = torch.empty(spec.n_ffn + 1, dtype=torch.int32, device=dev)
+    alpha = torch.empty(T, max(spec.n_const, 1), 2, device=dev)
+    ros = torch.empty(T, K, dtype=torch.int32, device=dev)
+    sor = torch.empty(cfg.M_cap, dtype=torch.int32, device=dev)
+    xp = torch.empty(cfg.M_cap, spec.D, dtype=td, device=dev)
+    hb = torch.empty(cfg.M_cap, spec.F, dtype=td, device=dev)
+    yp = torch.empty(cfg.M_cap, spec.D, dtype=td, device=dev)
+    yb = torch.empty_like(x0)
+    wd = wds[0]
+    p1 = prev0 if wd["W_g"] is not None else None
+    calls = [
+        ("route", lambda: B.moepp_route(cfg, x0, wd["W_r"], wd["W_g"], p1, wd["router_bias"], wd["W_c"], lgs[0], idx,
+                                        wk, cnt, off, alpha if spec.n_const else None)),
+        ("permute", lambda: B.moepp_permute(cfg, x0, idx, off, ros, sor, xp)),
+        ("grouped_ffn", lambda: B.moepp_grouped_ffn(cfg, xp, off, wd["W_gate"], wd["W_up"], wd["W_down"], hb, yp)),
+        ("combine", lambda: B.moepp_combine(cfg, x0, yp, idx, wk, ros, alpha if spec.n_const else None, wd["W_c"],
+                                            wd["v"], yb)),
+    ]
+    reps = max(5, args.steps)
+    acc = {n: 0.0 for n, _ in calls}
+    for it in range(3 + reps):
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(len(calls) + 1)]
+        evs[0].record()
+        for i, (_, fn) in enumerate(calls):
+            fn()
+            evs[i + 1].record()
+        torch.cuda.synchronize()
+        if it >= 3:
+            for i, (n, _) in enumerate(calls):
+                acc[n] += evs[i].elapsed_time(evs[i + 1]) / reps
+    counts = cnt.cpu().numpy()
+    M = int(off[-1].item())
+    zc_share = float(counts[spec.n_ffn:].sum()) / float(counts.sum())
+    es = 2 if spec.dtype == "bf16" else 4
+    flops_ffn = 6.0 * spec.D * spec.F * M
+    ffn_tflops = flops_ffn / (acc["grouped_ffn"] * 1e-3) / 1e12
+    # layer roofline: slower of FFN flops at the tensor peak and layer bytes at HBM bandwidth
+    active = int((counts[:spec.n_ffn] > 0).sum())
+    bytes_layer = (2.0 * T * spec.D * es + 3.0 * spec.D * spec.F * es * active + 4.0 * T * N * (2 if p1 is not None else 1)
+                   + 2.0 * M * spec.F * es)
+    t_roof_ms = max(flops_ffn / (peaks["burst"] * 1e12), bytes_layer / (peaks["hbm_gbs"] * 1e9)) * 1e3
+    layer_ms = ms_step / L
+
+    # ---- end to end through the host-buffer call --------------------------------------------------------------
+    xh = [x0.cpu().pin_memory()] + [torch.empty(T, spec.D, dtype=td).pin_memory() for _ in range(2)]
+    lh = [torch.empty(T, N).pin_memory() for _ in range(2)]
+    p0h = None if prev0 is None else prev0.cpu().pin_memory()
+
+    def step_host():
+        x, prev = xh[0], p0h
+        for j, w_ in enumerate(wds):
+            y, lg = xh[1 + (j & 1)], lh[j & 1]
+            B.moepp_layer_forward_host(cfg, w_, x, prev if w_["W_g"] is not None else None, y, lg, ws)
+            x, prev = y, lg
+        torch.cuda.current_stream().synchronize()  # the step's result is on the host
+
+    ms_e2e, _ = timed(step_host, max(3, args.steps // 4), 2)
+    act_b, lg_b = T * spec.D * es, T * N * 4
+    h2d = sum(act_b + (lg_b if w_["W_g"] is not None else 0) for w_ in wds)
+    d2h = L * (act_b + lg_b)
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+    cpu = None if args.no_cpu_baseline else cpu_baseline(args.workload)
+    key = WORKLOADS[args.workload][0]
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": key, "layers": L, "T": T, "D": spec.D, "F": spec.F,
+                   "experts": "%d+%d" % (spec.n_ffn, spec.n_zc), "top_k": K, "tokens_per_step_per_gpu": tokens_per_step,
+                   "zc_slot_share_layer1": round(zc_share, 4), "ffn_rows_layer1": M,
+                   "l2": "inputs larger than L2 (weights %.0f MB per layer); no explicit flush" %
+                         (3.0 * spec.D * spec.F * es * spec.n_ffn / 1e6),
+                   "parallelism": "replicas: each GPU runs its own token batch, no collective" if world > 1 else "1 GPU"},
+        "clocks": clocks,
+        "e2e": {"value": world * tokens_per_step / (ms_e2e * 1e-3), "unit": UNIT, "ms_per_step": ms_e2e,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "path": "moepp_layer_forward_host per layer, pinned host activations"},
+        "gpu_launches": args.steps * L * 7,
+        "roofline": {"kernel": "grouped_gemm_kernel (SwiGLU GEMM + down GEMM, 2 launches per layer)", "bound": "tensor",
+                     "achieved": ffn_tflops, "peak": peaks["sustained"], "unit": "TFLOP/s",
+                     "frac": ffn_tflops / peaks["sustained"], "peak_source": "bf16 sustained, of " + peaks["source"],
+                     "frac_of_burst_peak": ffn_tflops / peaks["burst"], "flops_per_call": flops_ffn,
+                     "ms_per_call": acc["grouped_ffn"], "traffic": None},
+        "layer_roofline": {"t_roof_ms": t_roof_ms, "t_layer_ms": layer_ms, "frac": t_roof_ms / layer_ms,
+                           "peaks": "bf16 burst %.1f TFLOP/s, HBM %.1f GB/s, of %s" % (peaks["burst"], peaks["hbm_gbs"],
+                                                                                         peaks["source"]),
+                           "roof_bytes": bytes_layer, "note": "first layer's routing; all layers timed"},
+        "breakdown_ms_layer1": {k: round(v, 4) for k, v in acc.items()},
+        "vanilla": {"value": world * tokens_per_step / (ms_van * 1e-3), "unit": UNIT, "ms_per_step": ms_van,
+                    "speedup_of_moepp": ms_van / ms_step,
+                    "what": "same library, same T, D, F, n_ffn, K, no zero-computation experts"},
+        "cpu_baseline": cpu,
+        "paper_context": "paper reports 1.1-2.1x expert forward throughput over vanilla MoE (A100 cluster, conditions "
+                         "unstated); context only",
+    }
+    print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
