@@ -115,7 +115,8 @@ moepp_status layer_on_device(const Dims& d, const Carve& c, const moepp_weights*
 
 moepp_status check_layer_args(const Dims& d, const moepp_weights* w, const void* x, const float* prev, const void* y,
                               const void* ws) {
-  if (w == nullptr || x == nullptr || y == nullptr || ws == nullptr) return MOEPP_ERR_INVALID_ARG;
+  if (w == nullptr || ws == nullptr) return MOEPP_ERR_INVALID_ARG;
+  if (d.T > 0 && (x == nullptr || y == nullptr)) return MOEPP_ERR_INVALID_ARG;
   if (d.flags & MOEPP_FLAG_LOGITS_GIVEN) return MOEPP_ERR_INVALID_ARG;  // a whole layer computes its own logits
   if (w->W_r == nullptr) return MOEPP_ERR_INVALID_ARG;
   if ((w->W_g == nullptr) != (prev == nullptr)) return MOEPP_ERR_INVALID_ARG;
@@ -171,9 +172,8 @@ moepp_status moepp_route(const moepp_config* cfg, const void* x, const float* W_
   Dims d;
   const moepp_status s = make_dims(cfg, &d);
   if (s != MOEPP_OK) return s;
-  if (logits == nullptr || topk_idx == nullptr || topk_w == nullptr || expert_counts == nullptr ||
-      expert_offsets == nullptr)
-    return MOEPP_ERR_INVALID_ARG;
+  if (expert_counts == nullptr || expert_offsets == nullptr) return MOEPP_ERR_INVALID_ARG;
+  if (d.T > 0 && (logits == nullptr || topk_idx == nullptr || topk_w == nullptr)) return MOEPP_ERR_INVALID_ARG;
   const bool given = (d.flags & MOEPP_FLAG_LOGITS_GIVEN) != 0;
   if (given) {
     W_r = nullptr; W_g = nullptr; prev_logits = nullptr; router_bias = nullptr;
@@ -184,7 +184,7 @@ moepp_status moepp_route(const moepp_config* cfg, const void* x, const float* W_
   if (d.n_const == 0) alpha = nullptr;
   if (alpha != nullptr && W_c == nullptr) return MOEPP_ERR_INVALID_ARG;
   const bool needs_x = !given || alpha != nullptr;
-  if (needs_x && x == nullptr) return MOEPP_ERR_INVALID_ARG;
+  if (needs_x && d.T > 0 && x == nullptr) return MOEPP_ERR_INVALID_ARG;
   if (!aligned16(x) || !aligned16(W_r) || !aligned16(W_c)) return MOEPP_ERR_ALIGN;
   return from_cuda(launch_route(d, x, W_r, W_g, prev_logits, router_bias, W_c, logits, topk_idx, topk_w,
                                 expert_counts, expert_offsets, alpha, static_cast<cudaStream_t>(stream)));
@@ -196,9 +196,9 @@ moepp_status moepp_permute(const moepp_config* cfg, const void* x, const int32_t
   Dims d;
   const moepp_status s = make_dims(cfg, &d);
   if (s != MOEPP_OK) return s;
-  if (x == nullptr || topk_idx == nullptr || expert_offsets == nullptr || row_of_slot == nullptr ||
-      slot_of_row == nullptr || x_perm == nullptr)
-    return MOEPP_ERR_INVALID_ARG;
+  if (expert_offsets == nullptr) return MOEPP_ERR_INVALID_ARG;
+  if (d.T > 0 && (x == nullptr || topk_idx == nullptr || row_of_slot == nullptr)) return MOEPP_ERR_INVALID_ARG;
+  if (d.M_cap > 0 && (slot_of_row == nullptr || x_perm == nullptr)) return MOEPP_ERR_INVALID_ARG;
   if (!aligned16(x) || !aligned16(x_perm)) return MOEPP_ERR_ALIGN;
   return from_cuda(launch_permute(d, x, topk_idx, expert_offsets, row_of_slot, slot_of_row, x_perm,
                                   static_cast<cudaStream_t>(stream)));
@@ -210,7 +210,8 @@ moepp_status moepp_grouped_ffn(const moepp_config* cfg, const void* x_perm, cons
   Dims d;
   const moepp_status s = make_dims(cfg, &d);
   if (s != MOEPP_OK) return s;
-  if (x_perm == nullptr || expert_offsets == nullptr || h_ws == nullptr || y_perm == nullptr)
+  if (expert_offsets == nullptr) return MOEPP_ERR_INVALID_ARG;
+  if (d.T > 0 && d.n_ffn > 0 && (x_perm == nullptr || h_ws == nullptr || y_perm == nullptr))
     return MOEPP_ERR_INVALID_ARG;
   if (d.n_ffn > 0 && (W_gate == nullptr || W_up == nullptr || W_down == nullptr)) return MOEPP_ERR_INVALID_ARG;
   if (!aligned16(x_perm) || !aligned16(W_gate) || !aligned16(W_up) || !aligned16(W_down) || !aligned16(h_ws) ||
@@ -226,9 +227,9 @@ moepp_status moepp_combine(const moepp_config* cfg, const void* x, const void* y
   Dims d;
   const moepp_status s = make_dims(cfg, &d);
   if (s != MOEPP_OK) return s;
-  if (x == nullptr || topk_idx == nullptr || topk_w == nullptr || row_of_slot == nullptr || y == nullptr)
+  if (d.T > 0 && (x == nullptr || topk_idx == nullptr || topk_w == nullptr || row_of_slot == nullptr || y == nullptr))
     return MOEPP_ERR_INVALID_ARG;
-  if (d.n_ffn > 0 && y_perm == nullptr) return MOEPP_ERR_INVALID_ARG;
+  if (d.T > 0 && d.n_ffn > 0 && y_perm == nullptr) return MOEPP_ERR_INVALID_ARG;
   if (d.n_const > 0 && (v == nullptr || (alpha == nullptr && W_c == nullptr))) return MOEPP_ERR_INVALID_ARG;
   if (!aligned16(x) || !aligned16(y_perm) || !aligned16(y) || !aligned16(v) || !aligned16(W_c))
     return MOEPP_ERR_ALIGN;

@@ -74,6 +74,11 @@ def test_null_config_and_null_outputs(lib):
     assert lib.moepp_permute(ctypes.byref(c), *([null] * 7)) == 1
     assert lib.moepp_grouped_ffn(ctypes.byref(c), *([null] * 8)) == 1
     assert lib.moepp_combine(ctypes.byref(c), *([null] * 10)) == 1
+    one = ctypes.c_void_p(256)  # a non-null stand-in: these calls must fail on the NEXT missing pointer, before any launch
+    assert lib.moepp_route(ctypes.byref(c), null, null, null, null, null, null, null, null, null, one, one, null,
+                           null) == 1
+    assert lib.moepp_permute(ctypes.byref(c), null, null, one, null, null, null, null) == 1
+    assert lib.moepp_grouped_ffn(ctypes.byref(c), null, one, null, null, null, null, null, null) == 1
     assert lib.moepp_layer_forward(ctypes.byref(c), *([null] * 6), ctypes.c_size_t(0), null) == 1
     assert lib.moepp_layer_forward_host(ctypes.byref(c), *([null] * 6), ctypes.c_size_t(0), null) == 1
     assert lib.moepp_device_error(None) == 1
