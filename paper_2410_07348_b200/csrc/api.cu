@@ -119,7 +119,7 @@ moepp_status check_layer_args(const Dims& d, const moepp_weights* w, const void*
   if (d.T > 0 && (x == nullptr || y == nullptr)) return MOEPP_ERR_INVALID_ARG;
   if (d.flags & MOEPP_FLAG_LOGITS_GIVEN) return MOEPP_ERR_INVALID_ARG;  // a whole layer computes its own logits
   if (w->W_r == nullptr) return MOEPP_ERR_INVALID_ARG;
-  if ((w->W_g == nullptr) != (prev == nullptr)) return MOEPP_ERR_INVALID_ARG;
+  if (d.T > 0 && (w->W_g == nullptr) != (prev == nullptr)) return MOEPP_ERR_INVALID_ARG;
   if (d.n_const > 0 && (w->W_c == nullptr || w->v == nullptr)) return MOEPP_ERR_INVALID_ARG;
   if (d.n_ffn > 0 && (w->W_gate == nullptr || w->W_up == nullptr || w->W_down == nullptr))
     return MOEPP_ERR_INVALID_ARG;
@@ -179,7 +179,7 @@ moepp_status moepp_route(const moepp_config* cfg, const void* x, const float* W_
     W_r = nullptr; W_g = nullptr; prev_logits = nullptr; router_bias = nullptr;
   } else {
     if (W_r == nullptr) return MOEPP_ERR_INVALID_ARG;
-    if ((W_g == nullptr) != (prev_logits == nullptr)) return MOEPP_ERR_INVALID_ARG;
+    if (d.T > 0 && (W_g == nullptr) != (prev_logits == nullptr)) return MOEPP_ERR_INVALID_ARG;
   }
   if (d.n_const == 0) alpha = nullptr;
   if (alpha != nullptr && W_c == nullptr) return MOEPP_ERR_INVALID_ARG;
