@@ -165,6 +165,36 @@ moepp_status moepp_layer_forward_host(const moepp_config* cfg, const moepp_weigh
                                       void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * moepp_grouped_ffn without a scratch argument.  (The paper has no counterpart to this call: it exists
+ * for the way this library is embedded, not for the method.)
+ *
+ * Who needs it: code that is handed input and output buffers and nothing else, and that may not
+ * create device memory itself -- for example an operator plugged into a serving runtime whose
+ * memory planner owns every byte of the GPU and offers the operator no workspace slot, or a
+ * latency-critical loop in which a device allocation (which can stall the whole device) is
+ * off limits.  Such a caller cannot supply the [M_cap, F] intermediate that moepp_grouped_ffn wants.
+ *
+ * Here the intermediate lives in a fixed array of MOEPP_STATIC_SCRATCH_BYTES bytes inside the
+ * library's device image.  Consequences a caller must know:
+ *   - every GPU that loads the library sets that many bytes aside until the process exits;
+ *   - M_cap * F * sizeof(element) must not exceed MOEPP_STATIC_SCRATCH_BYTES; a larger problem is
+ *     refused with MOEPP_ERR_WORKSPACE before anything is launched;
+ *   - the first call on each device looks up the array's device address (a one-time runtime query,
+ *     made with that device current); make that first call outside any stream capture;
+ *   - all calls, on all streams, share the one array, and it keeps whatever the previous call left
+ *     there.  Nothing in it has to start at zero (every row the second GEMM reads for a live output
+ *     row was written by the first GEMM of the same call), so it is not cleared; but two calls that
+ *     overlap on the GPU (different streams, or different host threads) race on it.  Serialise them.
+ *   - the call itself allocates nothing and frees nothing, like the rest of the library.
+ * Arguments, layouts, results and status codes are otherwise those of moepp_grouped_ffn.
+ */
+#define MOEPP_STATIC_SCRATCH_BYTES (32u << 20)
+moepp_status moepp_grouped_ffn_static(const moepp_config* cfg, const void* x_perm, const int32_t* expert_offsets,
+                                      const void* W_gate, const void* W_up, const void* W_down,
+                                      void* y_perm, /* [M_cap, D] out */
+                                      void* stream);
+
+/*
  * Device-side waits in the tensor-core kernels are bounded.  If one ever runs out, the kernel
  * stops early and records a non-zero code; this call copies the code to *code (host pointer),
  * clears it, and synchronises the device while doing so.  0 = no kernel gave up.

@@ -23,7 +23,8 @@ STATUS = {0: "MOEPP_OK", 1: "MOEPP_ERR_INVALID_ARG", 2: "MOEPP_ERR_UNSUPPORTED",
 
 EXPORTS = ("moepp_status_string", "moepp_workspace_bytes", "moepp_workspace_bytes_host", "moepp_route",
            "moepp_permute", "moepp_grouped_ffn", "moepp_combine", "moepp_layer_forward",
-           "moepp_layer_forward_host", "moepp_device_error")
+           "moepp_layer_forward_host", "moepp_device_error", "moepp_grouped_ffn_static")
+STATIC_SCRATCH_BYTES = 32 << 20
 
 
 class MoeppError(RuntimeError):
@@ -134,6 +135,14 @@ def moepp_grouped_ffn(cfg, x_perm, expert_offsets, W_gate, W_up, W_down, h_ws, y
     c = cfg.c()
     _check(lib().moepp_grouped_ffn(ctypes.byref(c), _p(x_perm), _p(expert_offsets), _p(W_gate), _p(W_up), _p(W_down),
                                    _p(h_ws), _p(y_perm), _stream()), "moepp_grouped_ffn")
+
+
+def moepp_grouped_ffn_static(cfg, x_perm, expert_offsets, W_gate, W_up, W_down, y_perm):
+    """moepp_grouped_ffn for callers that own no scratch memory: the intermediate sits in a fixed
+    STATIC_SCRATCH_BYTES array inside the library.  Calls share that array, so do not overlap them."""
+    c = cfg.c()
+    _check(lib().moepp_grouped_ffn_static(ctypes.byref(c), _p(x_perm), _p(expert_offsets), _p(W_gate), _p(W_up),
+                                          _p(W_down), _p(y_perm), _stream()), "moepp_grouped_ffn_static")
 
 
 def moepp_combine(cfg, x, y_perm, topk_idx, topk_w, row_of_slot, alpha, W_c, v, y):
