@@ -30,6 +30,11 @@ cudaError_t launch_route(const Dims& d, const void* x, const float* W_r, const f
                          const float* bias, const float* W_c, float* logits, int32_t* topk_idx, float* topk_w,
                          int32_t* counts, int32_t* offsets, float* alpha, cudaStream_t st);
 
+// bf16 router with the projection on the tensor cores; cudaErrorNotSupported when it does not apply.
+cudaError_t launch_route_tc(const Dims& d, const void* x, const float* W_r, const float* W_g, const float* prev,
+                            const float* bias, const float* W_c, float* logits, int32_t* topk_idx, float* topk_w,
+                            int32_t* counts, float* alpha, cudaStream_t st);
+
 cudaError_t launch_permute(const Dims& d, const void* x, const int32_t* topk_idx, const int32_t* offsets,
                            int32_t* row_of_slot, int32_t* slot_of_row, void* x_perm, cudaStream_t st);
 
@@ -46,6 +51,7 @@ cudaError_t launch_combine(const Dims& d, const void* x, const void* y_perm, con
 
 // Error word written by kernels whose bounded waits ran out (0 = fine).
 cudaError_t read_and_clear_device_error(int32_t* code);
+int32_t* device_error_word();  // device address of that word on the current device (nullptr on failure)
 
 // ---- small device helpers -----------------------------------------------------------------------
 __device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }

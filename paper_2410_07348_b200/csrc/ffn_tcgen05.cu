@@ -16,6 +16,7 @@
 #include <cuda.h>
 
 #include "common.cuh"
+#include "tc_common.cuh"
 
 namespace moepp {
 
@@ -28,6 +29,11 @@ cudaError_t read_and_clear_device_error(int32_t* code) {
   if (e != cudaSuccess) return e;
   const int32_t zero = 0;
   return cudaMemcpyToSymbol(g_device_error, &zero, sizeof(int32_t));
+}
+
+int32_t* device_error_word() {
+  void* p = nullptr;
+  return cudaGetSymbolAddress(&p, g_device_error) == cudaSuccess ? static_cast<int32_t*>(p) : nullptr;
 }
 
 namespace {
@@ -43,102 +49,8 @@ constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kThreads = 192;
 constexpr int kTmemCols = 512;
 constexpr int kSmemBytes = kStages * kStageBytes + 1024;  // + slack to align the ring to 1024 B
-constexpr long long kWaitCycles = 4000000000LL;           // about two seconds: far beyond any healthy wait
 
-// instruction descriptor: D = f32, A = B = bf16, both K-major, N = 256, M = 128
-constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((UMMA_N >> 3) << 17) | ((BM >> 4) << 24);
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-
-// Bounded wait.  Returns false if the CTA is giving up (this wait ran out, or another one did).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int code) {
-  long long t0 = 0;
-  for (uint32_t spin = 0;; ++spin) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (spin >= 1024u) {
-      if (spin == 1024u) t0 = clock64();
-      if (*abort_flag != 0) return false;
-      if (clock64() - t0 > kWaitCycles) {
-        *abort_flag = code;
-        atomicCAS(&g_device_error, 0, code);
-        return false;
-      }
-      __nanosleep(64);
-    }
-  }
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1)
-      : "memory");
-}
-
-// shared-memory matrix descriptor: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
-  d |= (uint64_t)1 << 16;             // leading byte offset (not used by swizzled K-major layouts)
-  d |= (uint64_t)(1024 >> 4) << 32;   // stride byte offset
-  d |= (uint64_t)1 << 46;             // descriptor version of this architecture
-  d |= (uint64_t)2 << 61;             // 128-byte swizzle
-  return d;
-}
-
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(kIdesc), "r"(accumulate)
-      : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-// 16 consecutive accumulator columns of this thread's TMEM lane
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr));
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-// Ties the loaded registers to a point after the wait, so that no use of them is scheduled before it.
-__device__ __forceinline__ void tmem_ld_pin(uint32_t (&r)[16]) {
-  asm volatile("" : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
-                    "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]),
-                    "+r"(r[15])
-               :
-               : "memory");
-}
+constexpr uint32_t kIdesc = umma_idesc_bf16(BM, UMMA_N);
 
 __device__ __forceinline__ float silu_mul(float g, float u) { return __fdividef(g, 1.f + __expf(-g)) * u; }
 
@@ -229,7 +141,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const int brow = ti.e * Nout + ti.n0;
         for (int kb = 0; kb < KB; ++kb, ++it) {
           const uint32_t s = it % kStages, ph = (it / kStages) & 1u;
-          if (!mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u, &abort_flag, 1)) { ok = false; break; }
+          if (!mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u, &abort_flag, 1, &g_device_error)) { ok = false; break; }
           const uint32_t full = smem_u32(&bar_full[s]);
           const uint32_t a_dst = ring + s * kStageBytes, b_dst = a_dst + kABytes;
           mbar_expect_tx(full, kStageBytes);
@@ -257,19 +169,19 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       bool ok = true;
       for (int L = blockIdx.x; L < total_tiles && ok; L += gridDim.x, ++tile_iter) {
         const uint32_t buf = tile_iter & 1u, tph = (tile_iter >> 1) & 1u;
-        if (!mbar_wait(smem_u32(&bar_tmem_empty[buf]), tph ^ 1u, &abort_flag, 2)) { ok = false; break; }
+        if (!mbar_wait(smem_u32(&bar_tmem_empty[buf]), tph ^ 1u, &abort_flag, 2, &g_device_error)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * UMMA_N;
         for (int kb = 0; kb < KB; ++kb, ++it) {
           const uint32_t s = it % kStages, ph = (it / kStages) & 1u;
-          if (!mbar_wait(smem_u32(&bar_full[s]), ph, &abort_flag, 3)) { ok = false; break; }
+          if (!mbar_wait(smem_u32(&bar_full[s]), ph, &abort_flag, 3, &g_device_error)) { ok = false; break; }
           tc_fence_after();
           const uint32_t a_addr = ring + s * kStageBytes, b_addr = a_addr + kABytes;
           const uint64_t adesc = make_smem_desc(a_addr), bdesc = make_smem_desc(b_addr);
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
             // advancing k by 16 elements = 32 bytes inside the 128-byte swizzle row: +2 in the address field
-            umma_bf16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), (kb | k) != 0 ? 1u : 0u);
+            umma_bf16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), kIdesc, (kb | k) != 0 ? 1u : 0u);
           }
           umma_commit(smem_u32(&bar_empty[s]));  // stage reusable once these MMAs have read it
         }
@@ -289,7 +201,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     for (int L = blockIdx.x; L < total_tiles && ok; L += gridDim.x, ++tile_iter) {
       const TileInfo ti = decode(L, e);
       const uint32_t buf = tile_iter & 1u, tph = (tile_iter >> 1) & 1u;
-      if (!mbar_wait(smem_u32(&bar_tmem_full[buf]), tph, &abort_flag, 4)) { ok = false; break; }
+      if (!mbar_wait(smem_u32(&bar_tmem_full[buf]), tph, &abort_flag, 4, &g_device_error)) { ok = false; break; }
       tc_fence_after();
       const int grow = ti.row0 + q * 32 + lane;
       const bool row_ok = grow < ti.row_end;
@@ -352,11 +264,14 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   }
 }
 
+}  // namespace
+
 // ---- host side: tensor maps ---------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+namespace {
 EncodeTiledFn encode_fn() {
   static EncodeTiledFn fn = nullptr;
   if (fn == nullptr) {
@@ -370,19 +285,20 @@ EncodeTiledFn encode_fn() {
 }
 
 // [rows, cols] bf16 row-major matrix, box = box_rows x 64 columns, 128-byte swizzle, zero fill outside
-bool make_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+}  // namespace
+
+bool make_bf16_tile_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
   EncodeTiledFn fn = encode_fn();
   if (fn == nullptr || rows == 0) return false;
   const cuuint64_t dims[2] = {cols, rows};
   const cuuint64_t strides[1] = {cols * 2};
-  const cuuint32_t box[2] = {(cuuint32_t)BK, box_rows};
+  const cuuint32_t box[2] = {64u, box_rows};
   const cuuint32_t estr[2] = {1, 1};
   return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-}  // namespace
 
 cudaError_t launch_ffn_tcgen05(const Dims& d, const void* x_perm, const int32_t* offsets, const void* W_gate,
                                const void* W_up, const void* W_down, void* h, void* y_perm, cudaStream_t st) {
@@ -395,11 +311,11 @@ cudaError_t launch_ffn_tcgen05(const Dims& d, const void* x_perm, const int32_t*
 
   CUtensorMap mA1, mG, mU, mA2, mD;
   const uint64_t rows = (uint64_t)d.M_cap;
-  if (!make_map(&mA1, x_perm, rows, (uint64_t)d.D, BM) ||
-      !make_map(&mG, W_gate, (uint64_t)d.n_ffn * d.F, (uint64_t)d.D, 128) ||
-      !make_map(&mU, W_up, (uint64_t)d.n_ffn * d.F, (uint64_t)d.D, 128) ||
-      !make_map(&mA2, h, rows, (uint64_t)d.F, BM) ||
-      !make_map(&mD, W_down, (uint64_t)d.n_ffn * d.D, (uint64_t)d.F, 256))
+  if (!make_bf16_tile_map(&mA1, x_perm, rows, (uint64_t)d.D, BM) ||
+      !make_bf16_tile_map(&mG, W_gate, (uint64_t)d.n_ffn * d.F, (uint64_t)d.D, 128) ||
+      !make_bf16_tile_map(&mU, W_up, (uint64_t)d.n_ffn * d.F, (uint64_t)d.D, 128) ||
+      !make_bf16_tile_map(&mA2, h, rows, (uint64_t)d.F, BM) ||
+      !make_bf16_tile_map(&mD, W_down, (uint64_t)d.n_ffn * d.D, (uint64_t)d.F, 256))
     return cudaErrorNotSupported;
 
   auto k1 = grouped_gemm_kernel<true>;

@@ -234,7 +234,14 @@ cudaError_t launch_route(const Dims& d, const void* x, const float* W_r, const f
                          int32_t* counts, int32_t* offsets, float* alpha, cudaStream_t st) {
   cudaError_t err = cudaMemsetAsync(counts, 0, sizeof(int32_t) * d.N, st);
   if (err != cudaSuccess) return err;
-  if (d.T > 0) {
+  bool done = false;
+  if (d.T > 0) {  // bf16 activations: projection on the tensor cores
+    err = launch_route_tc(d, x, W_r, W_g, prev, bias, W_c, logits, topk_idx, topk_w, counts,
+                          d.n_const > 0 ? alpha : nullptr, st);
+    if (err == cudaSuccess) done = true;
+    else if (err != cudaErrorNotSupported) return err;
+  }
+  if (d.T > 0 && !done) {
     const int R = d.N + ((alpha != nullptr) ? 2 * d.n_const : 0);
     err = (d.dtype == MOEPP_BF16)
               ? launch_route_x<__nv_bfloat16>(d, R, x, W_r, W_g, prev, bias, W_c, logits, topk_idx, topk_w, counts,
