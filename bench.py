@@ -188,7 +188,7 @@ def cpu_baseline(name, budget_s=15.0):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="moepp", choices=["moepp", "reference"])
     ap.add_argument("--workload", default="cfg4", choices=sorted(WORKLOADS))

@@ -21,7 +21,7 @@
  *     (FFN | zero | copy | constant).  Slot s = t*K + k is the k-th pick of token t.
  *   - `dtype` is the storage type of x, y, x_perm, h, y_perm and the FFN weights.
  *     Router weights, logits, gate weights, W_c, v and all accumulation are float.
- *   - Activation and FFN-weight pointers must be 16-byte aligned; D and F must be
+ *   - Activation, FFN-weight and topk_idx pointers must be 16-byte aligned; D and F must be
  *     multiples of 8 (MOEPP_ERR_ALIGN otherwise).
  *   - M_cap = T*K + n_ffn*(row_align-1) is the row capacity of the grouped buffers.
  *   - Errors are returned, never thrown: argument errors are found on the host before

@@ -199,7 +199,7 @@ moepp_status moepp_permute(const moepp_config* cfg, const void* x, const int32_t
   if (expert_offsets == nullptr) return MOEPP_ERR_INVALID_ARG;
   if (d.T > 0 && (x == nullptr || topk_idx == nullptr || row_of_slot == nullptr)) return MOEPP_ERR_INVALID_ARG;
   if (d.M_cap > 0 && (slot_of_row == nullptr || x_perm == nullptr)) return MOEPP_ERR_INVALID_ARG;
-  if (!aligned16(x) || !aligned16(x_perm)) return MOEPP_ERR_ALIGN;
+  if (!aligned16(x) || !aligned16(x_perm) || !aligned16(topk_idx)) return MOEPP_ERR_ALIGN;
   return from_cuda(launch_permute(d, x, topk_idx, expert_offsets, row_of_slot, slot_of_row, x_perm,
                                   static_cast<cudaStream_t>(stream)));
 }

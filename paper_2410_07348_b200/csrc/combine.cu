@@ -8,7 +8,8 @@ namespace {
 
 constexpr int kCombineThreads = 256;
 
-template <typename XT>
+// KMAX: compile-time bound on the picks per token (2 or kMaxTopK); U: column chunks per trip.
+template <typename XT, int KMAX, int U>
 __global__ void __launch_bounds__(kCombineThreads)
 combine_kernel(Dims dm, const XT* __restrict__ x, const XT* __restrict__ y_perm, const int32_t* __restrict__ topk_idx,
                const float* __restrict__ topk_w, const int32_t* __restrict__ row_of_slot,
@@ -31,10 +32,10 @@ combine_kernel(Dims dm, const XT* __restrict__ x, const XT* __restrict__ y_perm,
   }
   // coefficient of x, and per-pick coefficient of v for constant picks
   float cx = dm.add_residual ? 1.f : 0.f;
-  float cv[kMaxTopK], wk[kMaxTopK];
-  int vq[kMaxTopK], rows[kMaxTopK];
+  float cv[KMAX], wk[KMAX];
+  int vq[KMAX], rows[KMAX];
 #pragma unroll
-  for (int k = 0; k < kMaxTopK; ++k) {
+  for (int k = 0; k < KMAX; ++k) {
     cv[k] = 0.f; vq[k] = -1; rows[k] = -1; wk[k] = 0.f;
     if (k < K) {
       const int e = __shfl_sync(0xffffffffu, e_l, k);
@@ -83,36 +84,58 @@ combine_kernel(Dims dm, const XT* __restrict__ x, const XT* __restrict__ y_perm,
   }
 
   XT* yt = y + (size_t)t * D;
-  for (int d = lane * 8; d < D; d += 256) {
-    float acc[8];
+  // U column chunks (256 elements each) per trip: all row loads of a trip are issued before any is used,
+  // so a warp keeps up to U * (picks + 1) 16-byte loads in flight.
+  for (int d0 = lane * 8; d0 < D; d0 += 256 * U) {
+    float acc[U][8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) acc[i] = 0.f;
-    if (cx != 0.f) {
-      float xv[8];
-      Vec8<XT>::load(xt + d, xv);
+    for (int u = 0; u < U; ++u) {
+      const int d = d0 + 256 * u;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) acc[i] = cx * xv[i];
+      for (int i = 0; i < 8; ++i) acc[u][i] = 0.f;
+      if (d < D && cx != 0.f) {
+        float xv[8];
+        Vec8<XT>::load(xt + d, xv);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[u][i] = cx * xv[i];
+      }
     }
 #pragma unroll
-    for (int k = 0; k < kMaxTopK; ++k) {
+    for (int k = 0; k < KMAX; ++k) {
       if (k < K) {
         if (rows[k] >= 0) {
-          float yv[8];
-          Vec8<XT>::load(y_perm + (size_t)rows[k] * D + d, yv);
+          float yv[U][8];
 #pragma unroll
-          for (int i = 0; i < 8; ++i) acc[i] = fmaf(wk[k], yv[i], acc[i]);
+          for (int u = 0; u < U; ++u) {
+            const int d = d0 + 256 * u;
+            if (d < D) Vec8<XT>::load(y_perm + (size_t)rows[k] * D + d, yv[u]);
+          }
+#pragma unroll
+          for (int u = 0; u < U; ++u)
+#pragma unroll
+            for (int i = 0; i < 8; ++i) acc[u][i] = fmaf(wk[k], yv[u][i], acc[u][i]);
         } else if (vq[k] >= 0) {
-          const float* vp = v + (size_t)vq[k] * D + d;
-          const float4 a = __ldg(reinterpret_cast<const float4*>(vp));
-          const float4 b = __ldg(reinterpret_cast<const float4*>(vp + 4));
-          acc[0] = fmaf(cv[k], a.x, acc[0]); acc[1] = fmaf(cv[k], a.y, acc[1]);
-          acc[2] = fmaf(cv[k], a.z, acc[2]); acc[3] = fmaf(cv[k], a.w, acc[3]);
-          acc[4] = fmaf(cv[k], b.x, acc[4]); acc[5] = fmaf(cv[k], b.y, acc[5]);
-          acc[6] = fmaf(cv[k], b.z, acc[6]); acc[7] = fmaf(cv[k], b.w, acc[7]);
+#pragma unroll
+          for (int u = 0; u < U; ++u) {
+            const int d = d0 + 256 * u;
+            if (d < D) {
+              const float* vp = v + (size_t)vq[k] * D + d;
+              const float4 a = __ldg(reinterpret_cast<const float4*>(vp));
+              const float4 b = __ldg(reinterpret_cast<const float4*>(vp + 4));
+              acc[u][0] = fmaf(cv[k], a.x, acc[u][0]); acc[u][1] = fmaf(cv[k], a.y, acc[u][1]);
+              acc[u][2] = fmaf(cv[k], a.z, acc[u][2]); acc[u][3] = fmaf(cv[k], a.w, acc[u][3]);
+              acc[u][4] = fmaf(cv[k], b.x, acc[u][4]); acc[u][5] = fmaf(cv[k], b.y, acc[u][5]);
+              acc[u][6] = fmaf(cv[k], b.z, acc[u][6]); acc[u][7] = fmaf(cv[k], b.w, acc[u][7]);
+            }
+          }
         }
       }
     }
-    Vec8<XT>::store(yt + d, acc);
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int d = d0 + 256 * u;
+      if (d < D) Vec8<XT>::store(yt + d, acc[u]);
+    }
   }
 }
 
@@ -124,14 +147,18 @@ cudaError_t launch_combine(const Dims& d, const void* x, const void* y_perm, con
   if (d.T == 0) return cudaSuccess;
   const int tokens_per_block = kCombineThreads / 32;
   const unsigned grid = (unsigned)((d.T + tokens_per_block - 1) / tokens_per_block);
-  if (d.dtype == MOEPP_BF16)
-    combine_kernel<__nv_bfloat16><<<grid, kCombineThreads, 0, st>>>(
-        d, static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(y_perm), topk_idx, topk_w,
-        row_of_slot, alpha, W_c, v, static_cast<__nv_bfloat16*>(y));
-  else
-    combine_kernel<float><<<grid, kCombineThreads, 0, st>>>(d, static_cast<const float*>(x),
-                                                            static_cast<const float*>(y_perm), topk_idx, topk_w,
-                                                            row_of_slot, alpha, W_c, v, static_cast<float*>(y));
+#define MOEPP_COMBINE(XT, KMAX, U)                                                                             \
+  combine_kernel<XT, KMAX, U><<<grid, kCombineThreads, 0, st>>>(                                               \
+      d, static_cast<const XT*>(x), static_cast<const XT*>(y_perm), topk_idx, topk_w, row_of_slot, alpha, W_c, \
+      v, static_cast<XT*>(y))
+  if (d.dtype == MOEPP_BF16) {
+    if (d.K <= 2) MOEPP_COMBINE(__nv_bfloat16, 2, 4);
+    else MOEPP_COMBINE(__nv_bfloat16, kMaxTopK, 1);
+  } else {
+    if (d.K <= 2) MOEPP_COMBINE(float, 2, 2);
+    else MOEPP_COMBINE(float, kMaxTopK, 1);
+  }
+#undef MOEPP_COMBINE
   return cudaGetLastError();
 }
 

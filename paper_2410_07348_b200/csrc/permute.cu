@@ -1,5 +1,6 @@
 // Grouping of the FFN slots (zero-computation slots never get a row) and the row gather.
 //   rank kernel  : stable rank of every FFN slot inside its expert -> row_of_slot, slot_of_row
+//                  (up to 64 CTAs, each finds the rows before its slot range by counting them itself)
 //   gather kernel: x_perm[row] = x[slot / K], 16-byte vectors, one warp per row
 // The rank is deterministic (ascending slot id inside an expert): no atomics decide placement.
 #include "common.cuh"
@@ -9,21 +10,44 @@ namespace {
 
 constexpr int kRankThreads = 1024;
 constexpr int kRankWarps = kRankThreads / 32;
+constexpr int kRankSlotsPerCta = 2048;
+constexpr int kRankMaxCtas = 64;
 
-// One CTA.  Warp w owns a contiguous range of slots.  Pass 1 counts its slots per expert, a scan over
-// (expert, warp) turns the counts into first rows, pass 2 hands out rows in slot order.
+// CTA b owns the contiguous slot range [b*per_cta, (b+1)*per_cta).  Phase 0 counts, per FFN expert, the
+// slots that precede the range (a plain shared-memory histogram of topk_idx[0, begin)): every CTA finds its
+// own starting rows without any exchange between CTAs.  Then, inside the range, warp w owns a contiguous
+// sub-range: pass 1 counts its slots per expert, a scan over (expert, warp) turns the counts into first
+// rows, pass 2 hands out rows in slot order.
 __global__ void __launch_bounds__(kRankThreads)
-permute_rank_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ offsets, long long S, int n_ffn,
-                    int32_t* __restrict__ row_of_slot, int32_t* __restrict__ slot_of_row) {
+permute_rank_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ offsets, long long S,
+                    long long per_cta, int n_ffn, int32_t* __restrict__ row_of_slot,
+                    int32_t* __restrict__ slot_of_row) {
   __shared__ int base[kRankWarps][kMaxExperts];
+  __shared__ int before[kMaxExperts];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   for (int i = tid; i < kRankWarps * kMaxExperts; i += kRankThreads) (&base[0][0])[i] = 0;
+  if (tid < kMaxExperts) before[tid] = 0;
   __syncthreads();
 
-  long long per_warp = (S + kRankWarps - 1) / kRankWarps;
+  const long long c_begin = (long long)blockIdx.x * per_cta;
+  const long long c_end = (c_begin + per_cta < S) ? c_begin + per_cta : S;
+
+  // phase 0: slots before this CTA's range, per FFN expert (16 bytes per load)
+  {
+    const int4* v = reinterpret_cast<const int4*>(topk_idx);  // c_begin is a multiple of 4
+    for (long long i = tid; i < c_begin / 4; i += kRankThreads) {
+      const int4 q = __ldg(v + i);
+      if (q.x < n_ffn) atomicAdd(&before[q.x], 1);
+      if (q.y < n_ffn) atomicAdd(&before[q.y], 1);
+      if (q.z < n_ffn) atomicAdd(&before[q.z], 1);
+      if (q.w < n_ffn) atomicAdd(&before[q.w], 1);
+    }
+  }
+
+  long long per_warp = (per_cta + kRankWarps - 1) / kRankWarps;
   per_warp = (per_warp + 31) / 32 * 32;
-  const long long s_begin = (long long)warp * per_warp;
-  const long long s_end = (s_begin + per_warp < S) ? s_begin + per_warp : S;
+  const long long s_begin = c_begin + (long long)warp * per_warp;
+  const long long s_end = (s_begin + per_warp < c_end) ? s_begin + per_warp : c_end;
   const unsigned lt_mask = (1u << lane) - 1u;
 
   for (long long s0 = s_begin; s0 < s_end; s0 += 32) {
@@ -36,7 +60,7 @@ permute_rank_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __restr
   }
   __syncthreads();
   if (tid < n_ffn) {
-    int run = offsets[tid];
+    int run = offsets[tid] + before[tid];
     for (int w = 0; w < kRankWarps; ++w) {
       const int c = base[w][tid];
       base[w][tid] = run;
@@ -99,7 +123,13 @@ cudaError_t launch_permute(const Dims& d, const void* x, const int32_t* topk_idx
   }
   if (d.T == 0) return cudaSuccess;
   const long long S = (long long)d.T * d.K;
-  permute_rank_kernel<<<1, kRankThreads, 0, st>>>(topk_idx, offsets, S, d.n_ffn, row_of_slot, slot_of_row);
+  long long n_cta = (S + kRankSlotsPerCta - 1) / kRankSlotsPerCta;
+  if (n_cta > kRankMaxCtas) n_cta = kRankMaxCtas;
+  long long per_cta = (S + n_cta - 1) / n_cta;
+  per_cta = (per_cta + 1023) / 1024 * 1024;  // whole warps of 32 slots, and 16-byte loads in phase 0
+  n_cta = (S + per_cta - 1) / per_cta;
+  permute_rank_kernel<<<(unsigned)n_cta, kRankThreads, 0, st>>>(topk_idx, offsets, S, per_cta, d.n_ffn, row_of_slot,
+                                                                slot_of_row);
   cudaError_t err = cudaGetLastError();
   if (err != cudaSuccess || d.n_ffn == 0 || d.M_cap == 0) return err;
   const int rows_per_block = 8;

@@ -22,7 +22,6 @@ namespace {
 
 constexpr int kTileTokens = 128;
 constexpr int kBK = 64;
-constexpr int kStagesR = 3;
 constexpr int kThreadsR = 192;
 constexpr int kABytesR = kTileTokens * kBK * 2;
 
@@ -30,7 +29,8 @@ template <int RP>
 struct RouteTcSmem {
   static constexpr int kBSub = RP * 128;  // one weight term: RP rows of 64 bf16
   static constexpr int kStage = kABytesR + 3 * kBSub;
-  static constexpr int kRing = kStagesR * kStage;
+  static constexpr int kStages = (RP == 128) ? 2 : 3;  // 128 stacked rows: 64 KiB per stage
+  static constexpr int kRing = kStages * kStage;
 };
 
 __device__ __forceinline__ void named_barrier_128() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
@@ -43,6 +43,7 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, Dims dm, const float* _
                 float* __restrict__ topk_w, int32_t* __restrict__ counts, float* __restrict__ alpha,
                 int32_t* err_word) {
   using L = RouteTcSmem<RP>;
+  constexpr int kStagesR = L::kStages;
   constexpr uint32_t kIdesc = umma_idesc_bf16(kTileTokens, RP);
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar_full[kStagesR], bar_empty[kStagesR], bar_tmem_full, bar_drain;
