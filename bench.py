@@ -194,6 +194,7 @@ def main():
     ap.add_argument("--workload", default="cfg4", choices=sorted(WORKLOADS))
     ap.add_argument("--ref-tokens", type=int, default=64)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--flags", type=int, default=0, help="MOEPP_FLAG_* bits passed in the configuration")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "moepp" else args.warmup
 
@@ -223,8 +224,8 @@ def main():
     spec, layers = build_stack(args.workload, W, dev)
     L = len(layers)
     add_res = 1 if L > 1 else 0
-    cfg = B.config_from_spec(spec, add_residual=add_res)
-    cfg_v = B.config_from_spec(spec.vanilla(), add_residual=add_res)
+    cfg = B.config_from_spec(spec, add_residual=add_res, flags=args.flags)
+    cfg_v = B.config_from_spec(spec.vanilla(), add_residual=add_res, flags=args.flags)
     wds = [B.weights_from_tensors(lt, dev) for lt in layers]
     wds_v = [vanilla_weights(wd, spec) for wd in wds]
     x0 = layers[0].x

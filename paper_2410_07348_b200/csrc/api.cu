@@ -81,7 +81,8 @@ moepp_status ffn_dispatch(const Dims& d, const void* x_perm, const int32_t* offs
                           const void* W_up, const void* W_down, void* h, void* y_perm, cudaStream_t st) {
   if (d.n_ffn == 0 || d.T == 0) return MOEPP_OK;
   if (d.dtype == MOEPP_BF16 && !(d.flags & MOEPP_FLAG_SIMT_FFN)) {
-    const cudaError_t e = launch_ffn_tcgen05(d, x_perm, offsets, W_gate, W_up, W_down, h, y_perm, st);
+    const cudaError_t e = ((d.flags & MOEPP_FLAG_FFN_SINGLE_CTA) ? launch_ffn_tcgen05 : launch_ffn_tcgen05_pair)(
+        d, x_perm, offsets, W_gate, W_up, W_down, h, y_perm, st);
     if (e == cudaErrorNotSupported) return MOEPP_ERR_UNSUPPORTED;
     return from_cuda(e);
   }

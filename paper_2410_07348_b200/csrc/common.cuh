@@ -45,6 +45,10 @@ cudaError_t launch_ffn_simt(const Dims& d, const void* x_perm, const int32_t* of
 cudaError_t launch_ffn_tcgen05(const Dims& d, const void* x_perm, const int32_t* offsets, const void* W_gate,
                                const void* W_up, const void* W_down, void* h, void* y_perm, cudaStream_t st);
 
+// the same on CTA pairs (cta_group::2, 256 x 256 tiles)
+cudaError_t launch_ffn_tcgen05_pair(const Dims& d, const void* x_perm, const int32_t* offsets, const void* W_gate,
+                                    const void* W_up, const void* W_down, void* h, void* y_perm, cudaStream_t st);
+
 cudaError_t launch_combine(const Dims& d, const void* x, const void* y_perm, const int32_t* topk_idx,
                            const float* topk_w, const int32_t* row_of_slot, const float* alpha, const float* W_c,
                            const float* v, void* y, cudaStream_t st);

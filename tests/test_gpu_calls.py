@@ -185,7 +185,8 @@ def test_grouped_ffn_bf16_fma_path(oracle64, row_align):
 @pytest.mark.parametrize("shape", [dict(), dict(D=256, F=512), dict(T=1, D=64, F=64), dict(T=40, D=1024, F=136),
                                    dict(T=3000, D=512, F=1024, n_ffn=3)])
 def test_grouped_ffn_bf16_tensor_cores(oracle64, row_align, shape):
-    ffn_case(oracle64, "bf16", row_align=row_align, **shape)
+    ffn_case(oracle64, "bf16", row_align=row_align, **shape)  # CTA pairs, 256 x 256 tiles
+    ffn_case(oracle64, "bf16", row_align=row_align, flags=B.FLAG_FFN_SINGLE_CTA, **shape)  # single CTAs, 128 x 256
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
