@@ -106,10 +106,20 @@ moepp_status layer_on_device(const Dims& d, const Carve& c, const moepp_weights*
   cudaError_t e = launch_route(d, x, w->W_r, w->W_g, prev, w->router_bias, w->W_c, logits, topk_idx, topk_w, counts,
                                offsets, alpha, st);
   if (e != cudaSuccess) return MOEPP_ERR_CUDA;
-  e = launch_permute(d, x, topk_idx, offsets, row_of_slot, slot_of_row, x_perm, st);
+  // bf16 on tensor cores: GEMM 1 gathers its rows from x itself, so the grouped copy of x is never built
+  const bool fused_gather = d.dtype == MOEPP_BF16 && !(d.flags & (MOEPP_FLAG_SIMT_FFN | MOEPP_FLAG_STAGED_PERMUTE));
+  e = launch_permute(d, x, topk_idx, offsets, row_of_slot, slot_of_row, fused_gather ? nullptr : x_perm, st);
   if (e != cudaSuccess) return MOEPP_ERR_CUDA;
-  const moepp_status s = ffn_dispatch(d, x_perm, offsets, w->W_gate, w->W_up, w->W_down, h, y_perm, st);
-  if (s != MOEPP_OK) return s;
+  if (fused_gather) {
+    if (d.n_ffn > 0 && d.T > 0) {
+      e = launch_ffn_tcgen05_gather(d, x, slot_of_row, offsets, w->W_gate, w->W_up, w->W_down, h, y_perm, st);
+      if (e == cudaErrorNotSupported) return MOEPP_ERR_UNSUPPORTED;
+      if (e != cudaSuccess) return MOEPP_ERR_CUDA;
+    }
+  } else {
+    const moepp_status s = ffn_dispatch(d, x_perm, offsets, w->W_gate, w->W_up, w->W_down, h, y_perm, st);
+    if (s != MOEPP_OK) return s;
+  }
   e = launch_combine(d, x, y_perm, topk_idx, topk_w, row_of_slot, alpha, w->W_c, w->v, y, st);
   return from_cuda(e);
 }

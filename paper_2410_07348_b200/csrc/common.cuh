@@ -45,6 +45,11 @@ cudaError_t launch_ffn_simt(const Dims& d, const void* x_perm, const int32_t* of
 cudaError_t launch_ffn_tcgen05(const Dims& d, const void* x_perm, const int32_t* offsets, const void* W_gate,
                                const void* W_up, const void* W_down, void* h, void* y_perm, cudaStream_t st);
 
+// single-CTA kernels with GEMM 1 gathering its rows from x through slot_of_row (x_perm is never built)
+cudaError_t launch_ffn_tcgen05_gather(const Dims& d, const void* x, const int32_t* slot_of_row, const int32_t* offsets,
+                                      const void* W_gate, const void* W_up, const void* W_down, void* h, void* y_perm,
+                                      cudaStream_t st);
+
 // the same on CTA pairs (cta_group::2, 256 x 256 tiles)
 cudaError_t launch_ffn_tcgen05_pair(const Dims& d, const void* x_perm, const int32_t* offsets, const void* W_gate,
                                     const void* W_up, const void* W_down, void* h, void* y_perm, cudaStream_t st);

@@ -60,11 +60,16 @@ struct TileInfo {
 
 // SWIGLU: C has Nout columns, the tile covers 128 of them (gate | up in the accumulator).
 // otherwise the tile covers 256 columns of C.
-template <bool SWIGLU>
+// GATHER: the A rows are not read from a grouped buffer but fetched straight from the token-major
+// activations: row r of the tile is token slot_of_row[r] / K, loaded four rows at a time with TMA
+// gather loads (tmA then describes x with a one-row box); pad rows and rows beyond the rows in use
+// are pointed at row T, outside the tensor, and arrive as zeros.
+template <bool SWIGLU, bool GATHER>
 __global__ void __launch_bounds__(kThreads, 1)
 grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                     const __grid_constant__ CUtensorMap tmB1, __nv_bfloat16* __restrict__ C,
-                    const int32_t* __restrict__ offsets, int n_ffn, int Nout, int Kd) {
+                    const int32_t* __restrict__ offsets, int n_ffn, int Nout, int Kd,
+                    const int32_t* __restrict__ slot_of_row, int top_k, int n_tokens) {
   constexpr int BN_OUT = SWIGLU ? 128 : 256;
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar_full[kStages], bar_empty[kStages], bar_tmem_full[2], bar_tmem_empty[2],
@@ -129,32 +134,57 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
   if (warp == 0) {
     // ---------------------------------- TMA producer ---------------------------------------------
-    if (lane == 0) {
-      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
-      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB0) : "memory");
-      if (SWIGLU) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB1) : "memory");
+    // one lane issues tile loads; with GATHER all 32 lanes work: lane l fetches rows 4l..4l+3 of the A tile
+    if (GATHER || lane == 0) {
+      if (lane == 0) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB0) : "memory");
+        if (SWIGLU) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB1) : "memory");
+      }
       uint32_t it = 0;
       int e = 0;
       bool ok = true;
+      const int rows_in_use = seg_begin[n_ffn];
       for (int L = blockIdx.x; L < total_tiles && ok; L += gridDim.x) {
         const TileInfo ti = decode(L, e);
         const int brow = ti.e * Nout + ti.n0;
+        int tok[4] = {0, 0, 0, 0};
+        if (GATHER) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int r = ti.row0 + lane * 4 + i;
+            const int slot = (r < rows_in_use) ? __ldg(slot_of_row + r) : -1;
+            tok[i] = (slot >= 0) ? slot / top_k : n_tokens;  // row n_tokens lies outside x: zero fill
+          }
+        }
         for (int kb = 0; kb < KB; ++kb, ++it) {
           const uint32_t s = it % kStages, ph = (it / kStages) & 1u;
-          if (!mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u, &abort_flag, 1, &g_device_error)) { ok = false; break; }
+          bool got = mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u, &abort_flag, 1, &g_device_error);
+          if (GATHER) got = __all_sync(0xffffffffu, got);
+          if (!got) { ok = false; break; }
           const uint32_t full = smem_u32(&bar_full[s]);
           const uint32_t a_dst = ring + s * kStageBytes, b_dst = a_dst + kABytes;
-          mbar_expect_tx(full, kStageBytes);
-          tma_load_2d(a_dst, &tmA, kb * BK, ti.row0, full);
-          if (SWIGLU) {
-            tma_load_2d(b_dst, &tmB0, kb * BK, brow, full);
-            tma_load_2d(b_dst + kBBytes / 2, &tmB1, kb * BK, brow, full);
+          if (lane == 0) mbar_expect_tx(full, kStageBytes);
+          if (GATHER) {
+            asm volatile(
+                "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes "
+                "[%0], [%1, {%3, %4, %5, %6, %7}], [%2];" ::"r"(a_dst + (uint32_t)lane * 512u),
+                "l"(&tmA), "r"(full), "r"(kb * BK), "r"(tok[0]), "r"(tok[1]), "r"(tok[2]), "r"(tok[3])
+                : "memory");
           } else {
-            tma_load_2d(b_dst, &tmB0, kb * BK, brow, full);
+            tma_load_2d(a_dst, &tmA, kb * BK, ti.row0, full);
+          }
+          if (lane == 0) {
+            if (SWIGLU) {
+              tma_load_2d(b_dst, &tmB0, kb * BK, brow, full);
+              tma_load_2d(b_dst + kBBytes / 2, &tmB1, kb * BK, brow, full);
+            } else {
+              tma_load_2d(b_dst, &tmB0, kb * BK, brow, full);
+            }
           }
         }
       }
-      if (!ok) {  // give the copies already issued a bounded chance to land before the CTA leaves
+      if (!ok && lane == 0) {  // give the copies already issued a bounded chance to land before the CTA leaves
         const uint32_t n_back = it < (uint32_t)kStages ? it : (uint32_t)kStages;
         for (uint32_t i = 1; i <= n_back; ++i) {
           const uint32_t j = it - i, s = j % kStages, ph = (j / kStages) & 1u;
@@ -318,17 +348,55 @@ cudaError_t launch_ffn_tcgen05(const Dims& d, const void* x_perm, const int32_t*
       !make_bf16_tile_map(&mD, W_down, (uint64_t)d.n_ffn * d.D, (uint64_t)d.F, 256))
     return cudaErrorNotSupported;
 
-  auto k1 = grouped_gemm_kernel<true>;
-  auto k2 = grouped_gemm_kernel<false>;
+  auto k1 = grouped_gemm_kernel<true, false>;
+  auto k2 = grouped_gemm_kernel<false, false>;
   err = cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
   if (err != cudaSuccess) return err;
   err = cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
   if (err != cudaSuccess) return err;
 
-  k1<<<sms, kThreads, kSmemBytes, st>>>(mA1, mG, mU, static_cast<__nv_bfloat16*>(h), offsets, d.n_ffn, d.F, d.D);
+  k1<<<sms, kThreads, kSmemBytes, st>>>(mA1, mG, mU, static_cast<__nv_bfloat16*>(h), offsets, d.n_ffn, d.F, d.D,
+                                        nullptr, 1, 0);
   err = cudaGetLastError();
   if (err != cudaSuccess) return err;
-  k2<<<sms, kThreads, kSmemBytes, st>>>(mA2, mD, mD, static_cast<__nv_bfloat16*>(y_perm), offsets, d.n_ffn, d.D, d.F);
+  k2<<<sms, kThreads, kSmemBytes, st>>>(mA2, mD, mD, static_cast<__nv_bfloat16*>(y_perm), offsets, d.n_ffn, d.D, d.F,
+                                        nullptr, 1, 0);
+  return cudaGetLastError();
+}
+
+// The same FFN with GEMM 1 reading its rows straight from x through slot_of_row (no grouped copy of x).
+cudaError_t launch_ffn_tcgen05_gather(const Dims& d, const void* x, const int32_t* slot_of_row, const int32_t* offsets,
+                                      const void* W_gate, const void* W_up, const void* W_down, void* h, void* y_perm,
+                                      cudaStream_t st) {
+  if (d.T == 0 || d.n_ffn == 0 || d.M_cap == 0) return cudaSuccess;
+  int dev = 0, sms = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return err;
+  err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (err != cudaSuccess) return err;
+
+  CUtensorMap mX, mG, mU, mA2, mD;
+  const uint64_t rows = (uint64_t)d.M_cap;
+  if (!make_bf16_tile_map(&mX, x, (uint64_t)d.T, (uint64_t)d.D, 1) ||
+      !make_bf16_tile_map(&mG, W_gate, (uint64_t)d.n_ffn * d.F, (uint64_t)d.D, 128) ||
+      !make_bf16_tile_map(&mU, W_up, (uint64_t)d.n_ffn * d.F, (uint64_t)d.D, 128) ||
+      !make_bf16_tile_map(&mA2, h, rows, (uint64_t)d.F, BM) ||
+      !make_bf16_tile_map(&mD, W_down, (uint64_t)d.n_ffn * d.D, (uint64_t)d.F, 256))
+    return cudaErrorNotSupported;
+
+  auto k1 = grouped_gemm_kernel<true, true>;
+  auto k2 = grouped_gemm_kernel<false, false>;
+  err = cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  if (err != cudaSuccess) return err;
+  err = cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  if (err != cudaSuccess) return err;
+
+  k1<<<sms, kThreads, kSmemBytes, st>>>(mX, mG, mU, static_cast<__nv_bfloat16*>(h), offsets, d.n_ffn, d.F, d.D,
+                                        slot_of_row, d.K, d.T);
+  err = cudaGetLastError();
+  if (err != cudaSuccess) return err;
+  k2<<<sms, kThreads, kSmemBytes, st>>>(mA2, mD, mD, static_cast<__nv_bfloat16*>(y_perm), offsets, d.n_ffn, d.D, d.F,
+                                        nullptr, 1, 0);
   return cudaGetLastError();
 }
 

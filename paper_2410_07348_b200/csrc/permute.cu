@@ -131,7 +131,7 @@ cudaError_t launch_permute(const Dims& d, const void* x, const int32_t* topk_idx
   permute_rank_kernel<<<(unsigned)n_cta, kRankThreads, 0, st>>>(topk_idx, offsets, S, per_cta, d.n_ffn, row_of_slot,
                                                                 slot_of_row);
   cudaError_t err = cudaGetLastError();
-  if (err != cudaSuccess || d.n_ffn == 0 || d.M_cap == 0) return err;
+  if (err != cudaSuccess || d.n_ffn == 0 || d.M_cap == 0 || x_perm == nullptr) return err;  // nullptr: tables only
   const int rows_per_block = 8;
   const unsigned grid = (unsigned)((d.M_cap + rows_per_block - 1) / rows_per_block);
   if (d.dtype == MOEPP_BF16)
