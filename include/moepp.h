@@ -53,8 +53,8 @@ typedef enum { MOEPP_F32 = 0, MOEPP_BF16 = 1 } moepp_dtype;
 /* flags */
 #define MOEPP_FLAG_LOGITS_GIVEN 1 /* moepp_route reads `logits` instead of computing Eq. 2 / Eq. 6 */
 #define MOEPP_FLAG_SIMT_FFN 2     /* bf16 only: run the FFN on the plain FMA kernel (cross-check path) */
-#define MOEPP_FLAG_STAGED_PERMUTE 8 /* moepp_layer_forward, bf16: build x_perm and run the staged FFN instead of
-                                      letting GEMM 1 gather its rows from x */
+#define MOEPP_FLAG_FUSED_GATHER 8  /* moepp_layer_forward, bf16: GEMM 1 fetches its rows from x with TMA gather loads
+                                      and x_perm is never built (measured slower than the staged default on B200) */
 #define MOEPP_FLAG_FFN_SINGLE_CTA 4 /* bf16 only: 128x256 tiles on single CTAs instead of 256x256 on CTA pairs */
 
 typedef struct {

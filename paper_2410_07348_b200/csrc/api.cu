@@ -106,8 +106,8 @@ moepp_status layer_on_device(const Dims& d, const Carve& c, const moepp_weights*
   cudaError_t e = launch_route(d, x, w->W_r, w->W_g, prev, w->router_bias, w->W_c, logits, topk_idx, topk_w, counts,
                                offsets, alpha, st);
   if (e != cudaSuccess) return MOEPP_ERR_CUDA;
-  // bf16 on tensor cores: GEMM 1 gathers its rows from x itself, so the grouped copy of x is never built
-  const bool fused_gather = d.dtype == MOEPP_BF16 && !(d.flags & (MOEPP_FLAG_SIMT_FFN | MOEPP_FLAG_STAGED_PERMUTE));
+  // optional: GEMM 1 gathers its rows from x itself, so the grouped copy of x is never built
+  const bool fused_gather = d.dtype == MOEPP_BF16 && (d.flags & MOEPP_FLAG_FUSED_GATHER) && !(d.flags & MOEPP_FLAG_SIMT_FFN);
   e = launch_permute(d, x, topk_idx, offsets, row_of_slot, slot_of_row, fused_gather ? nullptr : x_perm, st);
   if (e != cudaSuccess) return MOEPP_ERR_CUDA;
   if (fused_gather) {

@@ -100,8 +100,8 @@ def test_cfg2_bf16(oracle64):
     assert 0.2 < info["zc_share"] < 0.5
     check_layer(oracle64, lt, 64, host=True)
     check_layer(oracle64, lt, 64, flags=B.FLAG_SIMT_FFN)
-    check_layer(oracle64, lt, 64, flags=B.FLAG_STAGED_PERMUTE)  # x_perm built, staged FFN on CTA pairs
-    check_layer(oracle64, lt, 64, flags=B.FLAG_STAGED_PERMUTE | B.FLAG_FFN_SINGLE_CTA)
+    check_layer(oracle64, lt, 64, flags=B.FLAG_FFN_SINGLE_CTA)  # 128 x 256 tiles on single CTAs
+    check_layer(oracle64, lt, 64, flags=B.FLAG_FUSED_GATHER)  # GEMM 1 gathers its rows from x
 
 
 def test_cfg3_bf16_skewed(oracle64):
