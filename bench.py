@@ -95,11 +95,12 @@ WORKLOADS = {  # name -> (config key, layers)
 }
 
 
-def build_stack(name, W, device):
+def build_stack(name, W, device, n_layers=0):
     """Layer tensors of the workload, generated on the device with seeded generators."""
-    key, n_layers = WORKLOADS[name]
+    key, full = WORKLOADS[name]
+    n_layers = min(n_layers, full) if n_layers > 0 else full
     spec = W.CONFIGS[key]
-    if n_layers > 1:
+    if full > 1:
         return spec, W.make_stack(spec, n_layers, device=device, gen_device=device)
     return spec, [W.make_config(key, device=device, gen_device=device)]
 
@@ -194,6 +195,7 @@ def main():
     ap.add_argument("--workload", default="cfg4", choices=sorted(WORKLOADS))
     ap.add_argument("--ref-tokens", type=int, default=64)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0, help="use only the first N layers of the workload (profiling)")
     ap.add_argument("--flags", type=int, default=0, help="MOEPP_FLAG_* bits passed in the configuration")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "moepp" else args.warmup
@@ -221,7 +223,7 @@ def main():
     B.lib()
 
     peaks = load_peaks()
-    spec, layers = build_stack(args.workload, W, dev)
+    spec, layers = build_stack(args.workload, W, dev, args.layers)
     L = len(layers)
     add_res = 1 if L > 1 else 0
     cfg = B.config_from_spec(spec, add_residual=add_res, flags=args.flags)
