@@ -8,9 +8,10 @@ namespace {
 
 constexpr int kCombineThreads = 256;
 
-// KMAX: compile-time bound on the picks per token (2 or kMaxTopK); U: column chunks per trip.
-template <typename XT, int KMAX, int U>
-__global__ void __launch_bounds__(kCombineThreads)
+// KMAX: compile-time bound on the picks per token (2 or kMaxTopK); U: column chunks per trip;
+// MINB: blocks per SM the register allocation must allow.
+template <typename XT, int KMAX, int U, int MINB>
+__global__ void __launch_bounds__(kCombineThreads, MINB)
 combine_kernel(Dims dm, const XT* __restrict__ x, const XT* __restrict__ y_perm, const int32_t* __restrict__ topk_idx,
                const float* __restrict__ topk_w, const int32_t* __restrict__ row_of_slot,
                const float* __restrict__ alpha, const float* __restrict__ W_c, const float* __restrict__ v,
@@ -147,12 +148,14 @@ cudaError_t launch_combine(const Dims& d, const void* x, const void* y_perm, con
   if (d.T == 0) return cudaSuccess;
   const int tokens_per_block = kCombineThreads / 32;
   const unsigned grid = (unsigned)((d.T + tokens_per_block - 1) / tokens_per_block);
-#define MOEPP_COMBINE(XT, KMAX, U)                                                                             \
-  combine_kernel<XT, KMAX, U><<<grid, kCombineThreads, 0, st>>>(                                               \
+#define MOEPP_COMBINE(XT, KMAX, U)  MOEPP_COMBINE2(XT, KMAX, U, 1)
+#define MOEPP_COMBINE2(XT, KMAX, U, MINB)                                                                             \
+  combine_kernel<XT, KMAX, U, MINB><<<grid, kCombineThreads, 0, st>>>(                                               \
       d, static_cast<const XT*>(x), static_cast<const XT*>(y_perm), topk_idx, topk_w, row_of_slot, alpha, W_c, \
       v, static_cast<XT*>(y))
   if (d.dtype == MOEPP_BF16) {
-    if (d.K <= 2) MOEPP_COMBINE(__nv_bfloat16, 2, 4);
+    // two chunks per trip at four blocks per SM (64 registers) keeps the most bytes in flight: measured best
+    if (d.K <= 2) MOEPP_COMBINE2(__nv_bfloat16, 2, 2, 4);
     else MOEPP_COMBINE(__nv_bfloat16, kMaxTopK, 1);
   } else {
     if (d.K <= 2) MOEPP_COMBINE(float, 2, 2);
