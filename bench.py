@@ -233,19 +233,16 @@ def main():
     x0 = layers[0].x
     prev0 = layers[0].prev
     prev0_v = None if prev0 is None else prev0[:, :spec.n_ffn].contiguous()
-    ws = torch.empty(max(B.moepp_workspace_bytes(cfg, host=True), B.moepp_workspace_bytes(cfg_v, host=True)),
-                     dtype=torch.uint8, device=dev)
-    xs = [torch.empty_like(x0) for _ in range(2)]
-    lgs = [torch.empty(spec.T, spec.N, device=dev) for _ in range(2)]
-    lgs_v = [torch.empty(spec.T, spec.n_ffn, device=dev) for _ in range(2)]
+    ws = torch.empty(max(B.moepp_stack_workspace_bytes(cfg, L, host=True), B.moepp_stack_workspace_bytes(cfg_v, L, host=True),
+                         B.moepp_workspace_bytes(cfg, host=True)), dtype=torch.uint8, device=dev)
+    y_out = torch.empty_like(x0)
+    lg_out = torch.empty(spec.T, spec.N, device=dev)
+    lg_out_v = torch.empty(spec.T, spec.n_ffn, device=dev)
+    lgs = [torch.empty(spec.T, spec.N, device=dev)]
 
-    def step(c, wlist, logit_bufs, p0):
-        x, prev = x0, p0
-        for j, wd in enumerate(wlist):
-            y, lg = xs[j & 1], logit_bufs[j & 1]
-            B.moepp_layer_forward(c, wd, x, prev if wd["W_g"] is not None else None, y, lg, ws)
-            x, prev = y, lg
-        return x
+    def step(c, wlist, lg, p0):
+        B.moepp_stack_forward(c, wlist, x0, p0 if wlist[0]["W_g"] is not None else None, y_out, lg, ws)
+        return y_out
 
     def timed(fn, steps, warmup, sampler=None):
         for _ in range(warmup):
@@ -271,13 +268,13 @@ def main():
 
     # ---- headline: the stack with inputs resident in HBM -------------------------------------------------
     sampler = ClockSampler(local_rank) if rank == 0 else None
-    ms_step, clocks = timed(lambda: step(cfg, wds, lgs, prev0), args.steps, args.warmup, sampler)
+    ms_step, clocks = timed(lambda: step(cfg, wds, lg_out, prev0), args.steps, args.warmup, sampler)
     assert B.moepp_device_error() == 0
     tokens_per_step = spec.T * L
     value = world * tokens_per_step / (ms_step * 1e-3)
 
     # ---- the same library as a vanilla all-FFN MoE of equal size ---------------------------------------------
-    ms_van, _ = timed(lambda: step(cfg_v, wds_v, lgs_v, prev0_v), max(3, args.steps // 2), 3)
+    ms_van, _ = timed(lambda: step(cfg_v, wds_v, lg_out_v, prev0_v), max(3, args.steps // 2), 3)
 
     # ---- per-call breakdown of layer 1 (staged calls, events between them) -----------------------------------
     T, N, K = spec.T, spec.N, spec.top_k
@@ -329,22 +326,19 @@ def main():
     layer_ms = ms_step / L
 
     # ---- end to end through the host-buffer call --------------------------------------------------------------
-    xh = [x0.cpu().pin_memory()] + [torch.empty(T, spec.D, dtype=td).pin_memory() for _ in range(2)]
-    lh = [torch.empty(T, N).pin_memory() for _ in range(2)]
-    p0h = None if prev0 is None else prev0.cpu().pin_memory()
+    xh = x0.cpu().pin_memory()
+    yh = torch.empty(T, spec.D, dtype=td).pin_memory()
+    lh = torch.empty(T, N).pin_memory()
+    p0h = None if (prev0 is None or wds[0]["W_g"] is None) else prev0.cpu().pin_memory()
 
     def step_host():
-        x, prev = xh[0], p0h
-        for j, w_ in enumerate(wds):
-            y, lg = xh[1 + (j & 1)], lh[j & 1]
-            B.moepp_layer_forward_host(cfg, w_, x, prev if w_["W_g"] is not None else None, y, lg, ws)
-            x, prev = y, lg
+        B.moepp_stack_forward_host(cfg, wds, xh, p0h, yh, lh, ws)
         torch.cuda.current_stream().synchronize()  # the step's result is on the host
 
     ms_e2e, _ = timed(step_host, max(3, args.steps // 4), 2)
     act_b, lg_b = T * spec.D * es, T * N * 4
-    h2d = sum(act_b + (lg_b if w_["W_g"] is not None else 0) for w_ in wds)
-    d2h = L * (act_b + lg_b)
+    h2d = act_b + (lg_b if p0h is not None else 0)
+    d2h = act_b + lg_b
 
     if rank != 0:
         if dist is not None:
@@ -365,7 +359,7 @@ def main():
         "clocks": clocks,
         "e2e": {"value": world * tokens_per_step / (ms_e2e * 1e-3), "unit": UNIT, "ms_per_step": ms_e2e,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "path": "moepp_layer_forward_host per layer, pinned host activations"},
+                "path": "moepp_stack_forward_host: x in and y, logits out through pinned host memory, layers chained on the device"},
         "gpu_launches": args.steps * L * 7,
         "roofline": {"kernel": "grouped_gemm_kernel (SwiGLU GEMM + down GEMM, 2 launches per layer)", "bound": "tensor",
                      "achieved": ffn_tflops, "peak": peaks["sustained"], "unit": "TFLOP/s",

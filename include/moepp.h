@@ -168,6 +168,26 @@ moepp_status moepp_layer_forward_host(const moepp_config* cfg, const moepp_weigh
                                       void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * A stack of n_layers layers that share one configuration (the gating residual of Eq. 6 carries the
+ * logits from layer to layer): layer j reads x^j and the logits of layer j-1 and produces
+ * x^{j+1} = (x^j if add_residual) + Eq. 1 and its own logits.  layers[j] holds layer j's weights; a layer
+ * whose W_g is NULL ignores the incoming logits (layer 1 of a model, Eq. 6 case j = 1).  prev_logits
+ * feeds layers[0] and may be NULL when layers[0].W_g is NULL.  y receives the last layer's output,
+ * logits_out (may be NULL) the last layer's logits.  Workspace: moepp_stack_workspace_bytes().
+ * The _host variant takes host pointers for x, prev_logits, y and logits_out (pinned memory for
+ * asynchronous copies): x goes to the device once, y comes back once, the layers in between stay on
+ * the device.  Workspace: moepp_stack_workspace_bytes_host().
+ */
+moepp_status moepp_stack_workspace_bytes(const moepp_config* cfg, int32_t n_layers, size_t* bytes);
+moepp_status moepp_stack_forward(const moepp_config* cfg, const moepp_weights* layers, int32_t n_layers, const void* x,
+                                 const float* prev_logits, void* y, float* logits_out, void* workspace,
+                                 size_t workspace_bytes, void* stream);
+moepp_status moepp_stack_workspace_bytes_host(const moepp_config* cfg, int32_t n_layers, size_t* bytes);
+moepp_status moepp_stack_forward_host(const moepp_config* cfg, const moepp_weights* layers, int32_t n_layers,
+                                      const void* x_host, const float* prev_logits_host, void* y_host,
+                                      float* logits_out_host, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * moepp_grouped_ffn without a scratch argument.  (The paper has no counterpart to this call: it exists
  * for the way this library is embedded, not for the method.)
  *

@@ -23,7 +23,9 @@ STATUS = {0: "MOEPP_OK", 1: "MOEPP_ERR_INVALID_ARG", 2: "MOEPP_ERR_UNSUPPORTED",
 
 EXPORTS = ("moepp_status_string", "moepp_workspace_bytes", "moepp_workspace_bytes_host", "moepp_route",
            "moepp_permute", "moepp_grouped_ffn", "moepp_combine", "moepp_layer_forward",
-           "moepp_layer_forward_host", "moepp_device_error", "moepp_grouped_ffn_static")
+           "moepp_layer_forward_host", "moepp_device_error", "moepp_grouped_ffn_static",
+           "moepp_stack_workspace_bytes", "moepp_stack_forward", "moepp_stack_workspace_bytes_host",
+           "moepp_stack_forward_host")
 STATIC_SCRATCH_BYTES = 32 << 20
 
 
@@ -165,6 +167,38 @@ def moepp_layer_forward_host(cfg, weights: dict, x_host, prev_logits_host, y_hos
                                           _p(y_host), _p(logits_out_host), _p(workspace),
                                           ctypes.c_size_t(workspace.numel() * workspace.element_size()), _stream()),
            "moepp_layer_forward_host")
+
+
+def _weights_array(weights_list):
+    arr = (moepp_weights * len(weights_list))()
+    for i, w in enumerate(weights_list):
+        arr[i] = _weights(w)
+    return arr
+
+
+def moepp_stack_workspace_bytes(cfg: Config, n_layers: int, host: bool = False) -> int:
+    n = ctypes.c_size_t(0)
+    c = cfg.c()
+    fn = lib().moepp_stack_workspace_bytes_host if host else lib().moepp_stack_workspace_bytes
+    _check(fn(ctypes.byref(c), ctypes.c_int32(n_layers), ctypes.byref(n)), "moepp_stack_workspace_bytes")
+    return int(n.value)
+
+
+def moepp_stack_forward(cfg, weights_list, x, prev_logits, y, logits_out, workspace):
+    c, arr = cfg.c(), _weights_array(weights_list)
+    _check(lib().moepp_stack_forward(ctypes.byref(c), arr, ctypes.c_int32(len(weights_list)), _p(x), _p(prev_logits),
+                                     _p(y), _p(logits_out), _p(workspace),
+                                     ctypes.c_size_t(workspace.numel() * workspace.element_size()), _stream()),
+           "moepp_stack_forward")
+
+
+def moepp_stack_forward_host(cfg, weights_list, x_host, prev_logits_host, y_host, logits_out_host, workspace):
+    """x_host, prev_logits_host, y_host, logits_out_host: pinned CPU tensors; weights and workspace: CUDA."""
+    c, arr = cfg.c(), _weights_array(weights_list)
+    _check(lib().moepp_stack_forward_host(ctypes.byref(c), arr, ctypes.c_int32(len(weights_list)), _p(x_host),
+                                          _p(prev_logits_host), _p(y_host), _p(logits_out_host), _p(workspace),
+                                          ctypes.c_size_t(workspace.numel() * workspace.element_size()), _stream()),
+           "moepp_stack_forward_host")
 
 
 def moepp_device_error() -> int:

@@ -296,6 +296,116 @@ moepp_status moepp_layer_forward_host(const moepp_config* cfg, const moepp_weigh
   return MOEPP_OK;
 }
 
+// Workspace of a stack: one layer workspace, two activation buffers and two logits buffers to ping-pong
+// between layers (plus, for host I/O, nothing more: the first activation buffer receives x).
+static size_t stack_extra_bytes(const Dims& d, size_t* act, size_t* lg) {
+  *act = align_up(elem_size(d.dtype) * (size_t)d.T * d.D + 1);
+  *lg = align_up(sizeof(float) * (size_t)d.T * d.N + 1);
+  return 2 * (*act) + 2 * (*lg);
+}
+
+moepp_status moepp_stack_workspace_bytes(const moepp_config* cfg, int32_t n_layers, size_t* bytes) {
+  Dims d;
+  const moepp_status s = make_dims(cfg, &d);
+  if (s != MOEPP_OK) return s;
+  if (bytes == nullptr || n_layers < 1) return MOEPP_ERR_INVALID_ARG;
+  size_t act, lg;
+  *bytes = carve(d, false).total + stack_extra_bytes(d, &act, &lg);
+  return MOEPP_OK;
+}
+
+static moepp_status stack_on_device(const Dims& d, const moepp_weights* layers, int32_t n_layers, const void* x,
+                                    const float* prev_logits, void* y, float* logits_out, char* ws, cudaStream_t st) {
+  const Carve c = carve(d, false);
+  size_t act, lg;
+  stack_extra_bytes(d, &act, &lg);
+  char* extra = ws + c.total;
+  void* xbuf[2] = {extra, extra + act};
+  float* lbuf[2] = {reinterpret_cast<float*>(extra + 2 * act), reinterpret_cast<float*>(extra + 2 * act + lg)};
+  const void* cur_x = x;
+  const float* cur_prev = prev_logits;
+  for (int j = 0; j < n_layers; ++j) {
+    const bool last = (j == n_layers - 1);
+    void* out_y = last ? y : xbuf[j & 1];
+    float* out_l = (last && logits_out != nullptr) ? logits_out : lbuf[j & 1];
+    const moepp_weights* w = &layers[j];
+    const float* prev = (w->W_g != nullptr) ? cur_prev : nullptr;
+    const moepp_status s = check_layer_args(d, w, cur_x, prev, out_y, ws);
+    if (s != MOEPP_OK) return s;
+    const moepp_status r = layer_on_device(d, c, w, cur_x, prev, out_y, out_l, ws, st);
+    if (r != MOEPP_OK) return r;
+    cur_x = out_y;
+    cur_prev = out_l;
+  }
+  return MOEPP_OK;
+}
+
+moepp_status moepp_stack_forward(const moepp_config* cfg, const moepp_weights* layers, int32_t n_layers, const void* x,
+                                 const float* prev_logits, void* y, float* logits_out, void* workspace,
+                                 size_t workspace_bytes, void* stream) {
+  Dims d;
+  const moepp_status s = make_dims(cfg, &d);
+  if (s != MOEPP_OK) return s;
+  if (layers == nullptr || n_layers < 1 || workspace == nullptr) return MOEPP_ERR_INVALID_ARG;
+  if (d.T > 0 && (x == nullptr || y == nullptr)) return MOEPP_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(y)) return MOEPP_ERR_ALIGN;
+  if ((reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) != 0) return MOEPP_ERR_ALIGN;
+  size_t act, lg;
+  if (workspace_bytes < carve(d, false).total + stack_extra_bytes(d, &act, &lg)) return MOEPP_ERR_WORKSPACE;
+  if (d.T > 0 && layers[0].W_g != nullptr && prev_logits == nullptr) return MOEPP_ERR_INVALID_ARG;
+  return stack_on_device(d, layers, n_layers, x, prev_logits, y, logits_out, static_cast<char*>(workspace),
+                         static_cast<cudaStream_t>(stream));
+}
+
+moepp_status moepp_stack_workspace_bytes_host(const moepp_config* cfg, int32_t n_layers, size_t* bytes) {
+  Dims d;
+  const moepp_status s = make_dims(cfg, &d);
+  if (s != MOEPP_OK) return s;
+  if (bytes == nullptr || n_layers < 1) return MOEPP_ERR_INVALID_ARG;
+  size_t act, lg;
+  const size_t extra = stack_extra_bytes(d, &act, &lg);
+  *bytes = carve(d, false).total + extra + 2 * act + 2 * lg;  // + staging of x, y, prev and the last logits
+  return MOEPP_OK;
+}
+
+moepp_status moepp_stack_forward_host(const moepp_config* cfg, const moepp_weights* layers, int32_t n_layers,
+                                      const void* x_host, const float* prev_logits_host, void* y_host,
+                                      float* logits_out_host, void* workspace, size_t workspace_bytes, void* stream) {
+  Dims d;
+  const moepp_status s = make_dims(cfg, &d);
+  if (s != MOEPP_OK) return s;
+  if (layers == nullptr || n_layers < 1 || workspace == nullptr) return MOEPP_ERR_INVALID_ARG;
+  if (d.T > 0 && (x_host == nullptr || y_host == nullptr)) return MOEPP_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) != 0) return MOEPP_ERR_ALIGN;
+  size_t act, lg;
+  const size_t extra = stack_extra_bytes(d, &act, &lg);
+  const size_t base = carve(d, false).total + extra;
+  if (workspace_bytes < base + 2 * act + 2 * lg) return MOEPP_ERR_WORKSPACE;
+  if (d.T > 0 && layers[0].W_g != nullptr && prev_logits_host == nullptr) return MOEPP_ERR_INVALID_ARG;
+  if (d.T == 0) return MOEPP_OK;
+  char* ws = static_cast<char*>(workspace);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char* x_dev = ws + base;
+  char* y_dev = x_dev + act;
+  float* p_dev = reinterpret_cast<float*>(y_dev + act);
+  float* l_dev = reinterpret_cast<float*>(y_dev + act + lg);
+  const size_t act_bytes = elem_size(d.dtype) * (size_t)d.T * d.D, lg_bytes = sizeof(float) * (size_t)d.T * d.N;
+  if (cudaMemcpyAsync(x_dev, x_host, act_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return MOEPP_ERR_CUDA;
+  const float* prev = nullptr;
+  if (prev_logits_host != nullptr) {
+    if (cudaMemcpyAsync(p_dev, prev_logits_host, lg_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+      return MOEPP_ERR_CUDA;
+    prev = p_dev;
+  }
+  const moepp_status r = stack_on_device(d, layers, n_layers, x_dev, prev, y_dev, l_dev, ws, st);
+  if (r != MOEPP_OK) return r;
+  if (cudaMemcpyAsync(y_host, y_dev, act_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return MOEPP_ERR_CUDA;
+  if (logits_out_host != nullptr &&
+      cudaMemcpyAsync(logits_out_host, l_dev, lg_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return MOEPP_ERR_CUDA;
+  return MOEPP_OK;
+}
+
 moepp_status moepp_device_error(int32_t* code) {
   if (code == nullptr) return MOEPP_ERR_INVALID_ARG;
   const cudaError_t e = read_and_clear_device_error(code);

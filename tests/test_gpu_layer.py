@@ -168,6 +168,54 @@ def test_cfg4_stack_of_four(oracle64):
         del lt, wd
 
 
+def test_stack_call_equals_chained_layer_calls(oracle64):
+    """moepp_stack_forward (and its host-buffer form) = the same layers called one after another."""
+    spec = W.LayerSpec(T=1500, D=512, F=768, n_ffn=6, dtype="bf16")
+    layers = W.make_stack(spec, 3, device="cuda", gen_device="cuda")
+    cfg = B.config_from_spec(spec, add_residual=1)
+    wds = [B.weights_from_tensors(lt) for lt in layers]
+    x = layers[0].x
+    ws = torch.empty(B.moepp_workspace_bytes(cfg), dtype=torch.uint8, device="cuda")
+    cur, prev = x, None
+    for wd in wds:
+        y = torch.empty_like(x)
+        lg = torch.empty(spec.T, spec.N, device="cuda")
+        B.moepp_layer_forward(cfg, wd, cur, prev if wd["W_g"] is not None else None, y, lg, ws)
+        cur, prev = y, lg
+    ws2 = torch.empty(B.moepp_stack_workspace_bytes(cfg, 3, host=True), dtype=torch.uint8, device="cuda")
+    y2 = torch.empty_like(x)
+    lg2 = torch.empty(spec.T, spec.N, device="cuda")
+    B.moepp_stack_forward(cfg, wds, x, None, y2, lg2, ws2)
+    torch.cuda.synchronize()
+    assert torch.equal(y2, cur) and torch.equal(lg2, prev)
+    xh, yh, lh = x.cpu().pin_memory(), torch.empty_like(x, device="cpu").pin_memory(), torch.empty(spec.T, spec.N).pin_memory()
+    B.moepp_stack_forward_host(cfg, wds, xh, None, yh, lh, ws2)
+    torch.cuda.synchronize()
+    assert torch.equal(yh.cuda(), cur) and torch.equal(lh.cuda(), prev)
+    assert B.moepp_device_error() == 0
+    # against the oracle: free-running chain on all tokens, following the GPU's picks layer by layer
+    s = shape_of(spec, add_residual=1)
+    x_o, prev_o = f32(x), None
+    cur, prev = x, None
+    for wd, lt in zip(wds, layers):
+        idx = torch.empty(spec.T, spec.top_k, dtype=torch.int32, device="cuda")
+        tmp = [torch.empty(spec.T, spec.top_k, device="cuda"), torch.empty(spec.N, dtype=torch.int32, device="cuda"),
+               torch.empty(spec.n_ffn + 1, dtype=torch.int32, device="cuda"), torch.empty(spec.T, spec.N, device="cuda")]
+        B.moepp_route(cfg, cur, wd["W_r"], wd["W_g"], prev if wd["W_g"] is not None else None, None, None, tmp[3], idx,
+                      tmp[0], tmp[1], tmp[2], None)
+        y = torch.empty_like(x)
+        lg = torch.empty(spec.T, spec.N, device="cuda")
+        B.moepp_layer_forward(cfg, wd, cur, prev if wd["W_g"] is not None else None, y, lg, ws)
+        torch.cuda.synchronize()
+        lt.x, lt.prev = None, None
+        oi = oracle_inputs(lt)
+        r = oracle64.layer_forward(s, x_o, oi["W_r"], oi["W_g"], prev_o if oi["W_g"] is not None else None, None,
+                                   oi["W_c"], oi["v"], oi["W_gate"], oi["W_up"], oi["W_down"],
+                                   forced_idx=idx.cpu().numpy())
+        assert rel_err_per_token(y.float().cpu().numpy(), r["y"]) <= BF16_REL_TOL
+        cur, prev, x_o, prev_o = y, lg, r["y"], r["logits"]
+
+
 def test_cfg4_teacher_forced_layers(oracle64):
     """Each layer of the stack fed the oracle's own state (rounded once to bf16): picks exact, outputs in tolerance."""
     spec = W.CONFIGS["cfg4_7b_stack"]
