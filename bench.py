@@ -29,6 +29,10 @@ sys.path.insert(0, ROOT)
 
 import torch  # noqa: E402
 
+# DRAM bytes (read + write) of one grouped-FFN call (GEMM 1 + GEMM 2 launches) from the ncu capture summarised in
+# profiles/layer_kernels_cfg4_one_layer.md; only valid for the CTA-pair kernels on the config-4 layer shape.
+NCU_FFN_TRAFFIC_BYTES = {"cfg4": 2591.0e6}
+
 METRIC = "moepp_expert_forward_tokens_per_s"
 UNIT = "tokens/s"
 
@@ -179,7 +183,7 @@ def cpu_baseline(name, budget_s=15.0):
 
     probe = 16
     dt = run(probe)
-    n_tok = int(max(probe, min(4096, budget_s / max(dt / probe, 1e-9))))
+    n_tok = int(max(probe, min(32768, budget_s / max(dt / probe, 1e-9))))
     dt = run(n_tok)
     return {"value": n_tok / dt, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
             "sample": "first layer of the workload on %d tokens (per-token cost does not depend on T), float "
@@ -361,11 +365,13 @@ def main():
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "path": "moepp_stack_forward_host: x in and y, logits out through pinned host memory, layers chained on the device"},
         "gpu_launches": args.steps * L * 7,
-        "roofline": {"kernel": "grouped_gemm_kernel (SwiGLU GEMM + down GEMM, 2 launches per layer)", "bound": "tensor",
+        "roofline": {"kernel": "grouped_gemm_pair_kernel (SwiGLU GEMM + down GEMM, 2 launches per layer)", "bound": "tensor",
                      "achieved": ffn_tflops, "peak": peaks["sustained"], "unit": "TFLOP/s",
                      "frac": ffn_tflops / peaks["sustained"], "peak_source": "bf16 sustained, of " + peaks["source"],
                      "frac_of_burst_peak": ffn_tflops / peaks["burst"], "flops_per_call": flops_ffn,
-                     "ms_per_call": acc["grouped_ffn"], "traffic": None},
+                     "ms_per_call": acc["grouped_ffn"],
+                     "traffic": NCU_FFN_TRAFFIC_BYTES.get(args.workload) if args.flags == 0 else None,
+                     "traffic_unit": "bytes per call (dram read + write, ncu)"},
         "layer_roofline": {"t_roof_ms": t_roof_ms, "t_layer_ms": layer_ms, "frac": t_roof_ms / layer_ms,
                            "peaks": "bf16 burst %.1f TFLOP/s, HBM %.1f GB/s, of %s" % (peaks["burst"], peaks["hbm_gbs"],
                                                                                          peaks["source"]),
