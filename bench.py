@@ -96,12 +96,16 @@ WORKLOADS = {  # name -> (config key, layers)
     "cfg4": ("cfg4_7b_stack", 4),
     "cfg3": ("cfg3_bf16_16e_skew", 1),
     "cfg2": ("cfg2_bf16_8e", 1),
+    "cfg5": ("cfg5_sweep", 1),  # with --tokens and --zc-share
 }
 
 
-def build_stack(name, W, device, n_layers=0):
+def build_stack(name, W, device, n_layers=0, tokens=0, zc_share=None):
     """Layer tensors of the workload, generated on the device with seeded generators."""
     key, full = WORKLOADS[name]
+    if name == "cfg5":
+        lt = W.make_config(key, device=device, gen_device=device, T=tokens or None, zc_share=zc_share)
+        return lt.spec, [lt]
     n_layers = min(n_layers, full) if n_layers > 0 else full
     spec = W.CONFIGS[key]
     if full > 1:
@@ -199,6 +203,8 @@ def main():
     ap.add_argument("--workload", default="cfg4", choices=sorted(WORKLOADS))
     ap.add_argument("--ref-tokens", type=int, default=64)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--tokens", type=int, default=0, help="cfg5: token count T")
+    ap.add_argument("--zc-share", type=float, default=0.3, help="cfg5: share of slots on zero-computation experts")
     ap.add_argument("--layers", type=int, default=0, help="use only the first N layers of the workload (profiling)")
     ap.add_argument("--flags", type=int, default=0, help="MOEPP_FLAG_* bits passed in the configuration")
     args = ap.parse_args()
@@ -227,7 +233,7 @@ def main():
     B.lib()
 
     peaks = load_peaks()
-    spec, layers = build_stack(args.workload, W, dev, args.layers)
+    spec, layers = build_stack(args.workload, W, dev, args.layers, args.tokens, args.zc_share)
     L = len(layers)
     add_res = 1 if L > 1 else 0
     cfg = B.config_from_spec(spec, add_residual=add_res, flags=args.flags)
