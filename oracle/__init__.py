@@ -41,7 +41,7 @@ def build(force: bool = False) -> str:
 class _Cfg(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "T", "D", "F", "n_ffn", "n_zero", "n_copy", "n_const", "top_k", "renorm_topk", "row_align",
-        "add_residual", "ffn_w_bf16")]
+        "add_residual", "ffn_w_bf16")] + [("tau", ctypes.c_float), ("capacity_factor", ctypes.c_float)]
 
 
 @dataclass
@@ -58,6 +58,8 @@ class LayerShape:
     renorm_topk: int = 0
     row_align: int = 1
     add_residual: int = 0
+    tau: float = 1.0  # Eq. 7 / Eq. 8
+    capacity_factor: float = 0.0  # Eq. 8 gamma; 0 = no limit
 
     @property
     def N(self) -> int:
@@ -110,7 +112,7 @@ class Oracle:
 
     def _cfg(self, s: LayerShape, ffn_w_bf16: int = 0):
         return ctypes.byref(_Cfg(s.T, s.D, s.F, s.n_ffn, s.n_zero, s.n_copy, s.n_const, s.top_k, s.renorm_topk,
-                                 s.row_align, s.add_residual, ffn_w_bf16))
+                                 s.row_align, s.add_residual, ffn_w_bf16, s.tau, s.capacity_factor))
 
     # Eq. 2 / Eq. 6
     def router_logits(self, s, x, W_r, W_g=None, prev=None, bias=None):
@@ -137,6 +139,19 @@ class Oracle:
         self._call("tables", self._cfg(s), _ptr(idx), _ptr(counts), _ptr(offsets), _ptr(row_of_slot),
                    _ptr(slot_of_row))
         return counts, offsets, row_of_slot, slot_of_row[:s.M_cap]
+
+    def capacities(self, s):
+        """(cap_ffn, cap_zc) of Eq. 8 in routing slots."""
+        a, b = ctypes.c_int32(0), ctypes.c_int32(0)
+        self._lib.oracle_capacities(self._cfg(s), ctypes.byref(a), ctypes.byref(b))
+        return int(a.value), int(b.value)
+
+    # Eq. 7
+    def balance_stats(self, s, G, idx):
+        G, idx = _f32(G), _i32(idx)
+        f, P, loss = np.empty(s.N, np.float32), np.empty(s.N, np.float32), np.empty(1, np.float32)
+        self._call("balance_stats", self._cfg(s), _ptr(G), _ptr(idx), _ptr(f), _ptr(P), _ptr(loss))
+        return f, P, float(loss[0])
 
     def permute_rows(self, s, x, slot_of_row):
         x, slot_of_row = _f32(x), _i32(slot_of_row)

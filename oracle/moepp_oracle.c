@@ -26,6 +26,19 @@ typedef ORACLE_REAL real;
 #define FN(name) CAT(ORACLE_PFX, name)
 
 #ifdef ORACLE_MAIN_TU
+void oracle_capacities(const oracle_config* c, int32_t* cap_ffn, int32_t* cap_zc) {
+  *cap_ffn = INT32_MAX;
+  *cap_zc = INT32_MAX;
+  if (c->capacity_factor <= 0.0f) return;
+  const double tau = c->tau > 0.0f ? (double)c->tau : 1.0;
+  const double slots = (double)c->T * (double)c->top_k;
+  const double denom = tau * c->n_ffn + (double)(c->n_zero + c->n_copy + c->n_const);
+  const double cf = ceil((double)c->capacity_factor * tau * slots / denom);
+  const double cz = ceil((double)c->capacity_factor * slots / denom);
+  *cap_ffn = cf > 2147483647.0 ? INT32_MAX : (int32_t)cf;
+  *cap_zc = cz > 2147483647.0 ? INT32_MAX : (int32_t)cz;
+}
+
 int oracle_num_threads(void) {
 #ifdef _OPENMP
   return omp_get_max_threads();
@@ -173,20 +186,30 @@ int FN(tables)(const oracle_config* c, const int32_t* idx, int32_t* counts, int3
     if (idx[s] < 0 || idx[s] >= N) return 2;
     counts[idx[s]] += 1;
   }
+  int32_t cap_ffn, cap_zc;
+  oracle_capacities(c, &cap_ffn, &cap_zc);
   offsets[0] = 0;
-  for (int e = 0; e < c->n_ffn; ++e) offsets[e + 1] = offsets[e] + ((counts[e] + A - 1) / A) * A;
+  for (int e = 0; e < c->n_ffn; ++e) {
+    const int kept = counts[e] < cap_ffn ? counts[e] : cap_ffn; /* Eq. 8: at most cap_ffn slots are served */
+    offsets[e + 1] = offsets[e] + ((kept + A - 1) / A) * A;
+  }
   if (!row_of_slot && !slot_of_row) return 0;
   if (slot_of_row)
     for (int64_t r = 0; r < M_cap; ++r) slot_of_row[r] = -1;
-  int32_t* seen = (int32_t*)calloc((size_t)(c->n_ffn > 0 ? c->n_ffn : 1), sizeof(int32_t));
-  for (int64_t s = 0; s < S; ++s) {
+  int32_t* seen = (int32_t*)calloc((size_t)N, sizeof(int32_t));
+  for (int64_t s = 0; s < S; ++s) { /* slot order = the order in which experts fill up */
     const int e = idx[s];
-    int32_t row = -1;
-    if (e < c->n_ffn) { /* zero-computation slots own no row */
+    const int32_t cap = e < c->n_ffn ? cap_ffn : cap_zc;
+    int32_t row;
+    if (seen[e] >= cap) {
+      row = -2; /* dropped */
+    } else if (e < c->n_ffn) {
       row = offsets[e] + seen[e];
-      seen[e] += 1;
       if (slot_of_row) slot_of_row[row] = (int32_t)s;
+    } else {
+      row = -1; /* zero-computation slots own no row */
     }
+    seen[e] += 1;
     if (row_of_slot) row_of_slot[s] = row;
   }
   free(seen);
@@ -289,7 +312,9 @@ int FN(combine)(const oracle_config* c, const float* x, const float* y_perm, con
         const int e = idx[(int64_t)t * K + k];
         const real g = (real)w[(int64_t)t * K + k];
         real contrib;
-        if (e < zero0) {
+        if (row_of_slot[(int64_t)t * K + k] == -2) {
+          contrib = 0; /* Eq. 8: dropped at a full expert */
+        } else if (e < zero0) {
           contrib = (real)y_perm[(int64_t)row_of_slot[(int64_t)t * K + k] * D + d];
         } else if (e < copy0) {
           contrib = 0; /* Eq. 3 */
@@ -338,6 +363,20 @@ int FN(layer_forward)(const oracle_config* c, const float* x, const float* W_r, 
     for (int k = 0; k < K; ++k) w[(int64_t)t * K + k] = (float)wt[k];
   }
 
+  /* Eq. 8: serve slots in slot order; a slot that finds its expert full is dropped */
+  int32_t cap_ffn, cap_zc;
+  oracle_capacities(c, &cap_ffn, &cap_zc);
+  char* dropped = (char*)calloc((size_t)c->T * K + 1, 1);
+  if (c->capacity_factor > 0.0f) {
+    int32_t seen[256];
+    memset(seen, 0, sizeof seen);
+    for (int64_t s = 0; s < (int64_t)c->T * K; ++s) {
+      const int e = idx[s];
+      if (seen[e] >= (e < zero0 ? cap_ffn : cap_zc)) dropped[s] = 1;
+      seen[e] += 1;
+    }
+  }
+
   const int n_out = tokens ? n_tokens : c->T;
 #pragma omp parallel
   {
@@ -355,6 +394,7 @@ int FN(layer_forward)(const oracle_config* c, const float* x, const float* W_r, 
         const int e = idx[(int64_t)t * K + k];
         /* the weight as stored (float), the same value the combine step is handed */
         const real g = (real)w[(int64_t)t * K + k];
+        if (dropped[(int64_t)t * K + k]) continue;
         if (e < zero0) {
           ffn_real(c, u, expert_w(W_gate, e, DF, c->ffn_w_bf16), expert_w(W_up, e, DF, c->ffn_w_bf16),
                    expert_w(W_down, e, DF, c->ffn_w_bf16), h, e_out);
@@ -374,5 +414,34 @@ int FN(layer_forward)(const oracle_config* c, const float* x, const float* W_r, 
     }
     free(buf);
   }
+  free(dropped);
+  return 0;
+}
+
+/* ---- Eq. 7: heterogeneous load-balance statistics ------------------------------------------------ */
+int FN(balance_stats)(const oracle_config* c, const float* G, const int32_t* idx, float* f, float* Pm,
+                      float* loss) {
+  if (bad_config(c) || !G || !idx || !f || !Pm || !loss) return 1;
+  const int N = n_experts(c), K = c->top_k;
+  if (N > 256) return 1;
+  const real tau = c->tau > 0.0f ? (real)c->tau : (real)1;
+  real fs[256], ps[256];
+  for (int i = 0; i < N; ++i) { fs[i] = 0; ps[i] = 0; }
+  for (int t = 0; t < c->T; ++t) {
+    real g[256], P[256];
+    for (int i = 0; i < N; ++i) g[i] = (real)G[(int64_t)t * N + i];
+    softmax_all(g, N, P);
+    for (int i = 0; i < N; ++i) ps[i] += P[i];
+    for (int k = 0; k < K; ++k) fs[idx[(int64_t)t * K + k]] += 1; /* token t selects this expert */
+  }
+  real L = 0;
+  for (int i = 0; i < N; ++i) {
+    const real fi = c->T > 0 ? fs[i] / (real)c->T : 0, pi = c->T > 0 ? ps[i] / (real)c->T : 0;
+    const real eta = i < c->n_ffn ? (real)1 : tau;
+    f[i] = (float)fi;
+    Pm[i] = (float)pi;
+    L += eta * fi * pi;
+  }
+  *loss = (float)L;
   return 0;
 }

@@ -29,7 +29,10 @@
  *     pre-softmax logits.
  *   - each constant expert owns its own W_c (2 x D) and v (D).
  *   - the FFN expert is a bias-free SwiGLU: W_down (silu(W_gate x) * (W_up x)).
- *   - no capacity limit, no token dropping (Eq. 8 is a pre-training device).
+ *   - no capacity limit unless capacity_factor > 0.  With a limit (Eq. 8), slots are served in slot
+ *     order (token-major, then pick order); a slot that arrives at a full expert is dropped: it
+ *     contributes nothing to y (the token passes on through the residual stream), owns no row
+ *     (row_of_slot = -2) and causes no FFN work.  expert_counts stay the selection counts.
  *
  * Parity pins: see tests/test_oracle_*.py.  No function here is unpinned.
  */
@@ -50,7 +53,15 @@ typedef struct {
   int32_t row_align;    /* each FFN expert's row segment is padded to a multiple of this (>= 1) */
   int32_t add_residual; /* 1: y = x + Eq. 1 (used only when layers are stacked) */
   int32_t ffn_w_bf16;   /* 0: FFN weights are float; 1: they are bf16 bit patterns (uint16_t) */
+  float tau;            /* Eq. 7 / Eq. 8: weight of the zero-computation experts; <= 0 means 1 */
+  float capacity_factor; /* Eq. 8 gamma; <= 0: no capacity limit (nothing is dropped) */
 } oracle_config;
+
+/* Eq. 8 with T read as the number of routing slots T*K (for K = 1 the printed formula), rounded up:
+ *   FFN expert:              ceil(gamma * tau * T*K / (tau * N_FFN + N_ZC))
+ *   zero-computation expert: ceil(gamma *       T*K / (tau * N_FFN + N_ZC))
+ * Both are INT32_MAX when capacity_factor <= 0. */
+void oracle_capacities(const oracle_config* c, int32_t* cap_ffn, int32_t* cap_zc);
 
 int oracle_num_threads(void);
 
@@ -60,7 +71,7 @@ int oracle_num_threads(void);
                        const float* W_g, const float* prev, const float* bias, float* G);          \
   /* Eq. 1 gate: softmax over all N, top-K on logits.  P_out may be NULL. */                       \
   int P##gate_topk(const oracle_config* c, const float* G, int32_t* idx, float* w, float* P_out);  \
-  /* Grouping tables for FFN slots only. */                                                        \
+  /* Grouping tables for FFN slots only.  row_of_slot: row | -1 (zero-computation slot) | -2 (dropped, Eq. 8). */                                                        \
   int P##tables(const oracle_config* c, const int32_t* idx, int32_t* counts, int32_t* offsets,     \
                 int32_t* row_of_slot, int32_t* slot_of_row);                                       \
   /* x_perm[row] = x[slot_of_row[row] / K]; rows with slot -1 are set to 0. */                     \
@@ -79,6 +90,10 @@ int oracle_num_threads(void);
   int P##combine(const oracle_config* c, const float* x, const float* y_perm, const int32_t* idx,  \
                  const float* w, const int32_t* row_of_slot, const float* alpha, const float* v,   \
                  float* y);                                                                        \
+  /* Eq. 7: f[i] = share of tokens that select expert i, P[i] = mean softmax weight of expert i,            \
+     loss = sum_i eta_i f[i] P[i] with eta = 1 (FFN) or tau (zero-computation). */                           \
+  int P##balance_stats(const oracle_config* c, const float* G, const int32_t* idx, float* f, float* Pm,     \
+                       float* loss);                                                                        \
   /* Whole layer by the definition, token by token, without any grouping.                          \
      tokens==NULL: all T tokens, y is [T,D]; else y is [n_tokens,D] for the listed tokens.         \
      forced_idx (may be NULL) replaces the top-K choice; the weights still come from the           \
