@@ -27,6 +27,13 @@
  *   - Errors are returned, never thrown: argument errors are found on the host before
  *     anything is launched; MOEPP_ERR_CUDA wraps a failed launch.  T == 0 is valid and does nothing.
  *   - Limits: N <= 64, 1 <= K <= min(N, 8), N + 2*n_const <= 128.
+ *   - Expert capacity (Eq. 8), only when capacity_factor > 0: with S = T*K routing slots an FFN expert
+ *     serves at most ceil(gamma*tau*S / (tau*n_ffn + n_zc)) slots and a zero-computation expert at most
+ *     ceil(gamma*S / (tau*n_ffn + n_zc)) (Eq. 8 with its T read as the number of routing slots; for K = 1
+ *     it is the printed formula).  Slots are served in slot order; a slot that arrives at a full expert
+ *     is dropped: row_of_slot = -2, no grouped row, no FFN work, no contribution to y (the token passes
+ *     on through the residual stream).  expert_counts always are the selection counts; expert_offsets
+ *     count served slots only.
  */
 #ifndef MOEPP_H
 #define MOEPP_H
@@ -66,6 +73,8 @@ typedef struct {
   int32_t row_align;                      /* 1: dense grouped layout; >1: pad each expert's rows to a multiple */
   int32_t add_residual;                   /* 0: y is Eq. 1; 1: y = x + Eq. 1 (for stacking layers) */
   int32_t flags;                          /* MOEPP_FLAG_* */
+  float tau;                              /* Eq. 7 / Eq. 8: weight of the zero-computation experts; <= 0 means 1 */
+  float capacity_factor;                  /* Eq. 8 gamma; <= 0 (default): no capacity limit, nothing is dropped */
 } moepp_config;
 
 typedef struct {
@@ -108,7 +117,8 @@ moepp_status moepp_route(const moepp_config* cfg, const void* x, const float* W_
 /*
  * Grouping of the FFN slots only; zero-computation slots get no row (the efficiency argument of the
  * paper's Section 3.4 made literal).  Rows are expert-major and, inside an expert, ascend in slot id.
- *   row_of_slot[s] = grouped row of slot s, or -1 for a zero-computation slot
+ *   row_of_slot[s] = grouped row of slot s, or -1 for a zero-computation slot, or -2 for a slot dropped
+ *                    at a full expert (Eq. 8; never without capacity_factor)
  *   slot_of_row[r] = slot held by row r, or -1 for a pad row / a row beyond expert_offsets[n_ffn]
  *   x_perm[r,:]    = x[slot_of_row[r] / K, :]; pad rows inside a segment are zero-filled; rows at or
  *                    beyond expert_offsets[n_ffn] are left untouched.
@@ -166,6 +176,17 @@ moepp_status moepp_workspace_bytes_host(const moepp_config* cfg, size_t* bytes);
 moepp_status moepp_layer_forward_host(const moepp_config* cfg, const moepp_weights* weights, const void* x_host,
                                       const float* prev_logits_host, void* y_host, float* logits_out_host,
                                       void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Heterogeneous load-balance statistics (Eq. 7), by-products of the router:
+ *   f[i] = expert_counts[i] / T   share of tokens that select expert i (sums to K)
+ *   P[i] = (1/T) sum_t Softmax(logits[t,:])_i
+ *   *loss = sum_i eta_i f[i] P[i],  eta_i = 1 for FFN experts and tau for zero-computation experts.
+ * f, P ([N] each) and loss ([1]) are device pointers.  The reduction order is fixed: results are
+ * reproducible from run to run.
+ */
+moepp_status moepp_balance_stats(const moepp_config* cfg, const float* logits, const int32_t* expert_counts, float* f,
+                                 float* P, float* loss, void* stream);
 
 /*
  * A stack of n_layers layers that share one configuration (the gating residual of Eq. 6 carries the

@@ -25,7 +25,7 @@ EXPORTS = ("moepp_status_string", "moepp_workspace_bytes", "moepp_workspace_byte
            "moepp_permute", "moepp_grouped_ffn", "moepp_combine", "moepp_layer_forward",
            "moepp_layer_forward_host", "moepp_device_error", "moepp_grouped_ffn_static",
            "moepp_stack_workspace_bytes", "moepp_stack_forward", "moepp_stack_workspace_bytes_host",
-           "moepp_stack_forward_host")
+           "moepp_stack_forward_host", "moepp_balance_stats")
 STATIC_SCRATCH_BYTES = 32 << 20
 
 
@@ -38,7 +38,7 @@ class MoeppError(RuntimeError):
 class moepp_config(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "T", "D", "F", "n_ffn", "n_zero", "n_copy", "n_const", "top_k", "dtype", "renorm_topk", "row_align",
-        "add_residual", "flags")]
+        "add_residual", "flags")] + [("tau", ctypes.c_float), ("capacity_factor", ctypes.c_float)]
 
 
 class moepp_weights(ctypes.Structure):
@@ -74,6 +74,8 @@ class Config:
     row_align: int = 1
     add_residual: int = 0
     flags: int = 0
+    tau: float = 1.0
+    capacity_factor: float = 0.0
 
     @property
     def N(self):
@@ -85,7 +87,8 @@ class Config:
 
     def c(self):
         return moepp_config(self.T, self.D, self.F, self.n_ffn, self.n_zero, self.n_copy, self.n_const, self.top_k,
-                            self.dtype, self.renorm_topk, self.row_align, self.add_residual, self.flags)
+                            self.dtype, self.renorm_topk, self.row_align, self.add_residual, self.flags, self.tau,
+                            self.capacity_factor)
 
 
 def _p(t):
@@ -169,6 +172,12 @@ def moepp_layer_forward_host(cfg, weights: dict, x_host, prev_logits_host, y_hos
            "moepp_layer_forward_host")
 
 
+def moepp_balance_stats(cfg, logits, expert_counts, f, P, loss):
+    c = cfg.c()
+    _check(lib().moepp_balance_stats(ctypes.byref(c), _p(logits), _p(expert_counts), _p(f), _p(P), _p(loss),
+                                     _stream()), "moepp_balance_stats")
+
+
 def _weights_array(weights_list):
     arr = (moepp_weights * len(weights_list))()
     for i, w in enumerate(weights_list):
@@ -198,7 +207,7 @@ def moepp_stack_forward_host(cfg, weights_list, x_host, prev_logits_host, y_host
     _check(lib().moepp_stack_forward_host(ctypes.byref(c), arr, ctypes.c_int32(len(weights_list)), _p(x_host),
                                           _p(prev_logits_host), _p(y_host), _p(logits_out_host), _p(workspace),
                                           ctypes.c_size_t(workspace.numel() * workspace.element_size()), _stream()),
-           "moepp_stack_forward_host")
+           "moepp_stack_forward_host", "moepp_balance_stats")
 
 
 def moepp_device_error() -> int:

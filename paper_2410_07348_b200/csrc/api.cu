@@ -1,5 +1,6 @@
 // C-ABI layer: argument validation on the host, workspace carving, and the five calls of the layer.
 // Nothing here allocates memory or synchronises the stream.
+#include <cmath>
 #include <cstring>
 
 #include "common.cuh"
@@ -35,6 +36,16 @@ moepp_status make_dims(const moepp_config* c, Dims* d) {
   d->dtype = c->dtype; d->renorm = c->renorm_topk ? 1 : 0; d->row_align = c->row_align;
   d->add_residual = c->add_residual ? 1 : 0; d->flags = c->flags;
   d->M_cap = M_cap;
+  d->tau = c->tau > 0.f ? c->tau : 1.f;
+  d->cap_on = c->capacity_factor > 0.f ? 1 : 0;
+  d->cap_ffn = d->cap_zc = 0x7fffffff;
+  if (d->cap_on) {  // Eq. 8 over the T*K routing slots, rounded up
+    const double denom = (double)d->tau * c->n_ffn + (double)(c->n_zero + c->n_copy + c->n_const);
+    const double cf = ceil((double)c->capacity_factor * d->tau * (double)S / denom);
+    const double cz = ceil((double)c->capacity_factor * (double)S / denom);
+    d->cap_ffn = cf > 2147483647.0 ? 0x7fffffff : (int)cf;
+    d->cap_zc = cz > 2147483647.0 ? 0x7fffffff : (int)cz;
+  }
   return MOEPP_OK;
 }
 
@@ -404,6 +415,16 @@ moepp_status moepp_stack_forward_host(const moepp_config* cfg, const moepp_weigh
       cudaMemcpyAsync(logits_out_host, l_dev, lg_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
     return MOEPP_ERR_CUDA;
   return MOEPP_OK;
+}
+
+moepp_status moepp_balance_stats(const moepp_config* cfg, const float* logits, const int32_t* expert_counts, float* f,
+                                 float* P, float* loss, void* stream) {
+  Dims d;
+  const moepp_status s = make_dims(cfg, &d);
+  if (s != MOEPP_OK) return s;
+  if (expert_counts == nullptr || f == nullptr || P == nullptr || loss == nullptr) return MOEPP_ERR_INVALID_ARG;
+  if (d.T > 0 && logits == nullptr) return MOEPP_ERR_INVALID_ARG;
+  return from_cuda(launch_balance_stats(d, logits, expert_counts, f, P, loss, static_cast<cudaStream_t>(stream)));
 }
 
 moepp_status moepp_device_error(int32_t* code) {

@@ -42,7 +42,9 @@ combine_kernel(Dims dm, const XT* __restrict__ x, const XT* __restrict__ y_perm,
       const int e = __shfl_sync(0xffffffffu, e_l, k);
       const float g = __shfl_sync(0xffffffffu, w_l, k);
       const int row = __shfl_sync(0xffffffffu, row_l, k);
-      if (e < zero0) {
+      if (row == -2) {
+        // Eq. 8: dropped at a full expert, contributes nothing
+      } else if (e < zero0) {
         rows[k] = row; wk[k] = g;
       } else if (e < copy0) {
         // Eq. 3: contributes nothing

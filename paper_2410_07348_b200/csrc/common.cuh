@@ -18,6 +18,9 @@ struct Dims {
   int n_ffn, n_zero, n_copy, n_const, N, K;
   int dtype, renorm, row_align, add_residual, flags;
   long long M_cap;
+  float tau;             // Eq. 7 / Eq. 8
+  int cap_on;            // Eq. 8 active
+  int cap_ffn, cap_zc;   // slots an FFN / a zero-computation expert serves (INT_MAX when off)
   __host__ __device__ int zero0() const { return n_ffn; }
   __host__ __device__ int copy0() const { return n_ffn + n_zero; }
   __host__ __device__ int const0() const { return n_ffn + n_zero + n_copy; }
@@ -53,6 +56,9 @@ cudaError_t launch_ffn_tcgen05_gather(const Dims& d, const void* x, const int32_
 // the same on CTA pairs (cta_group::2, 256 x 256 tiles)
 cudaError_t launch_ffn_tcgen05_pair(const Dims& d, const void* x_perm, const int32_t* offsets, const void* W_gate,
                                     const void* W_up, const void* W_down, void* h, void* y_perm, cudaStream_t st);
+
+cudaError_t launch_balance_stats(const Dims& d, const float* logits, const int32_t* counts, float* f, float* P,
+                                 float* loss, cudaStream_t st);
 
 cudaError_t launch_combine(const Dims& d, const void* x, const void* y_perm, const int32_t* topk_idx,
                            const float* topk_w, const int32_t* row_of_slot, const float* alpha, const float* W_c,

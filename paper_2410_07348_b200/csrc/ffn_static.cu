@@ -71,7 +71,8 @@ extern "C" moepp_status moepp_grouped_ffn_static(const moepp_config* c, const vo
     return MOEPP_ERR_ALIGN;
   if (c->T == 0 || c->n_ffn == 0) return MOEPP_OK;
 
-  Dims d;
+  Dims d{};
+  d.tau = 1.f; d.cap_on = 0; d.cap_ffn = d.cap_zc = 0x7fffffff;
   d.T = c->T; d.D = c->D; d.F = c->F;
   d.n_ffn = c->n_ffn; d.n_zero = c->n_zero; d.n_copy = c->n_copy; d.n_const = c->n_const;
   d.N = (int)N; d.K = c->top_k;

@@ -20,13 +20,19 @@ constexpr int kRankMaxCtas = 64;
 // rows, pass 2 hands out rows in slot order.
 __global__ void __launch_bounds__(kRankThreads)
 permute_rank_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ offsets, long long S,
-                    long long per_cta, int n_ffn, int32_t* __restrict__ row_of_slot,
-                    int32_t* __restrict__ slot_of_row) {
-  __shared__ int base[kRankWarps][kMaxExperts];
+                    long long per_cta, int n_ffn, int n_rank, int cap_ffn, int cap_zc,
+                    int32_t* __restrict__ row_of_slot, int32_t* __restrict__ slot_of_row) {
+  // n_rank: experts whose slots are ranked: the FFN experts, or all experts when a capacity limit (Eq. 8)
+  // is active, because then the zero-computation experts fill up and drop slots too.
+  __shared__ int base[kRankWarps][kMaxExperts];  // running rank (slots of this expert seen so far)
   __shared__ int before[kMaxExperts];
+  __shared__ int seg0[kMaxExperts];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   for (int i = tid; i < kRankWarps * kMaxExperts; i += kRankThreads) (&base[0][0])[i] = 0;
-  if (tid < kMaxExperts) before[tid] = 0;
+  if (tid < kMaxExperts) {
+    before[tid] = 0;
+    seg0[tid] = (tid < n_ffn) ? offsets[tid] : 0;
+  }
   __syncthreads();
 
   const long long c_begin = (long long)blockIdx.x * per_cta;
@@ -37,10 +43,10 @@ permute_rank_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __restr
     const int4* v = reinterpret_cast<const int4*>(topk_idx);  // c_begin is a multiple of 4
     for (long long i = tid; i < c_begin / 4; i += kRankThreads) {
       const int4 q = __ldg(v + i);
-      if (q.x < n_ffn) atomicAdd(&before[q.x], 1);
-      if (q.y < n_ffn) atomicAdd(&before[q.y], 1);
-      if (q.z < n_ffn) atomicAdd(&before[q.z], 1);
-      if (q.w < n_ffn) atomicAdd(&before[q.w], 1);
+      if (q.x < n_rank) atomicAdd(&before[q.x], 1);
+      if (q.y < n_rank) atomicAdd(&before[q.y], 1);
+      if (q.z < n_rank) atomicAdd(&before[q.z], 1);
+      if (q.w < n_rank) atomicAdd(&before[q.w], 1);
     }
   }
 
@@ -53,14 +59,14 @@ permute_rank_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __restr
   for (long long s0 = s_begin; s0 < s_end; s0 += 32) {
     const long long s = s0 + lane;
     int e = (s < s_end) ? topk_idx[s] : -1;
-    if (e >= n_ffn) e = -1;
+    if (e >= n_rank) e = -1;
     const unsigned peers = __match_any_sync(0xffffffffu, e);
     if (e >= 0 && (peers & lt_mask) == 0) base[warp][e] += __popc(peers);
     __syncwarp();
   }
   __syncthreads();
-  if (tid < n_ffn) {
-    int run = offsets[tid] + before[tid];
+  if (tid < n_rank) {
+    int run = before[tid];
     for (int w = 0; w < kRankWarps; ++w) {
       const int c = base[w][tid];
       base[w][tid] = run;
@@ -72,10 +78,14 @@ permute_rank_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __restr
     const long long s = s0 + lane;
     const bool live = s < s_end;
     int e = live ? topk_idx[s] : -1;
-    if (e >= n_ffn) e = -1;
+    if (e >= n_rank) e = -1;
     const unsigned peers = __match_any_sync(0xffffffffu, e);
-    int row = -1;
-    if (e >= 0) row = base[warp][e] + __popc(peers & lt_mask);
+    int row = -1;  // zero-computation slot: no row
+    if (e >= 0) {
+      const int rank = base[warp][e] + __popc(peers & lt_mask);
+      if (rank >= (e < n_ffn ? cap_ffn : cap_zc)) row = -2;  // Eq. 8: the expert is full, the slot is dropped
+      else if (e < n_ffn) row = seg0[e] + rank;
+    }
     __syncwarp();
     if (e >= 0 && (peers & lt_mask) == 0) base[warp][e] += __popc(peers);
     __syncwarp();
@@ -128,8 +138,9 @@ cudaError_t launch_permute(const Dims& d, const void* x, const int32_t* topk_idx
   long long per_cta = (S + n_cta - 1) / n_cta;
   per_cta = (per_cta + 1023) / 1024 * 1024;  // whole warps of 32 slots, and 16-byte loads in phase 0
   n_cta = (S + per_cta - 1) / per_cta;
-  permute_rank_kernel<<<(unsigned)n_cta, kRankThreads, 0, st>>>(topk_idx, offsets, S, per_cta, d.n_ffn, row_of_slot,
-                                                                slot_of_row);
+  permute_rank_kernel<<<(unsigned)n_cta, kRankThreads, 0, st>>>(topk_idx, offsets, S, per_cta, d.n_ffn,
+                                                                d.cap_on ? d.N : d.n_ffn, d.cap_ffn, d.cap_zc,
+                                                                row_of_slot, slot_of_row);
   cudaError_t err = cudaGetLastError();
   if (err != cudaSuccess || d.n_ffn == 0 || d.M_cap == 0 || x_perm == nullptr) return err;  // nullptr: tables only
   const int rows_per_block = 8;

@@ -180,14 +180,15 @@ route_kernel(Dims dm, const XT* __restrict__ x, const float* __restrict__ W_r, c
   if (tid < N && s_cnt[tid] != 0) atomicAdd(&counts[tid], s_cnt[tid]);
 }
 
-// offsets[e] = first row of FFN expert e; every segment is its count rounded up to row_align.
+// offsets[e] = first row of FFN expert e; every segment is its served count rounded up to row_align.
 __global__ void route_offsets_kernel(const int32_t* __restrict__ counts, int32_t* __restrict__ offsets, int n_ffn,
-                                     int row_align) {
+                                     int row_align, int cap_ffn) {
   if (threadIdx.x == 0 && blockIdx.x == 0) {
     int run = 0;
     offsets[0] = 0;
     for (int e = 0; e < n_ffn; ++e) {
-      run += (counts[e] + row_align - 1) / row_align * row_align;
+      const int served = counts[e] < cap_ffn ? counts[e] : cap_ffn;  // Eq. 8: a full expert serves no more
+      run += (served + row_align - 1) / row_align * row_align;
       offsets[e + 1] = run;
     }
   }
@@ -250,7 +251,7 @@ cudaError_t launch_route(const Dims& d, const void* x, const float* W_r, const f
                                       st);
     if (err != cudaSuccess) return err;
   }
-  route_offsets_kernel<<<1, 32, 0, st>>>(counts, offsets, d.n_ffn, d.row_align);
+  route_offsets_kernel<<<1, 32, 0, st>>>(counts, offsets, d.n_ffn, d.row_align, d.cap_ffn);
   return cudaGetLastError();
 }
 

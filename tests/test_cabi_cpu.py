@@ -82,6 +82,9 @@ def test_null_config_and_null_outputs(lib):
     assert lib.moepp_layer_forward(ctypes.byref(c), *([null] * 6), ctypes.c_size_t(0), null) == 1
     assert lib.moepp_layer_forward_host(ctypes.byref(c), *([null] * 6), ctypes.c_size_t(0), null) == 1
     assert lib.moepp_device_error(None) == 1
+    assert lib.moepp_balance_stats(ctypes.byref(c), *([null] * 6)) == 1
+    assert lib.moepp_stack_forward(ctypes.byref(c), null, 1, *([null] * 5), ctypes.c_size_t(0), null) == 1
+    assert lib.moepp_stack_forward_host(ctypes.byref(c), null, 1, *([null] * 5), ctypes.c_size_t(0), null) == 1
 
 
 def test_missing_library_is_a_hard_error(monkeypatch):

@@ -60,7 +60,8 @@ def check_layer(oracle64, lt, n_sample, host=False, **over):
     wd = B.weights_from_tensors(lt)
     x, prev = lt.x.cuda(), None if lt.prev is None else lt.prev.cuda()
     y, logits, idx_g, counts = gpu_layer(cfg, wd, x, prev, host=host)
-    s, oi = shape_of(spec, **{k: v for k, v in over.items() if k in ("renorm_topk", "row_align", "add_residual")}), \
+    s, oi = shape_of(spec, **{k: v for k, v in over.items()
+                              if k in ("renorm_topk", "row_align", "add_residual", "tau", "capacity_factor")}), \
         oracle_inputs(lt)
     toks = None if n_sample is None else sample_tokens(idx_g, spec.N, n_sample)
     r = oracle64.layer_forward(s, oi["x"], oi["W_r"], oi["W_g"], oi["prev"], oi["bias"], oi["W_c"], oi["v"],
@@ -272,3 +273,69 @@ def test_empty_and_degenerate(oracle64):
     for k in (1, 4):
         spec = W.LayerSpec(T=200, D=128, F=256, n_ffn=6, top_k=k, dtype="bf16")
         check_layer(oracle64, W.make_layer(spec, seed=3), None)
+
+
+@pytest.mark.parametrize("gamma,tau", [(1.1, 0.75), (0.6, 0.5), (8.0, 0.75)])
+def test_capacity_limited_layer(oracle64, gamma, tau):
+    """Eq. 8: slots beyond an expert's capacity are dropped in slot order (no row, no FFN work, no contribution)."""
+    spec = W.LayerSpec(T=3000, D=256, F=384, n_ffn=6, dtype="bf16")
+    lt = W.make_layer(spec, seed=21)
+    lt.bias = torch.tensor([0.8, 0.0, -0.2, 0.0, 0.0, 0.0, 0.6, 0.0, 0.0, 0.0])  # crowd FFN expert 0 and the zero expert
+    info = check_layer(oracle64, lt, None, tau=tau, capacity_factor=gamma)
+    check_layer(oracle64, lt, None, tau=tau, capacity_factor=gamma, row_align=128, add_residual=1)
+    # tables of the capacity-limited permutation, bit-exact
+    cfg = B.config_from_spec(spec, tau=tau, capacity_factor=gamma)
+    s = shape_of(spec, tau=tau, capacity_factor=gamma)
+    oi = oracle_inputs(lt)
+    G = oracle64.router_logits(s, oi["x"], oi["W_r"], oi["W_g"], oi["prev"], oi["bias"])
+    idx_o, _ = oracle64.gate_topk(s, G)
+    counts_o, offsets_o, ros_o, sor_o = oracle64.tables(s, idx_o)
+    d = lambda a: torch.from_numpy(a).cuda()
+    lg = d(G)
+    idx = torch.empty(spec.T, 2, dtype=torch.int32, device="cuda")
+    w = torch.empty(spec.T, 2, device="cuda")
+    cnt = torch.empty(spec.N, dtype=torch.int32, device="cuda")
+    off = torch.empty(spec.n_ffn + 1, dtype=torch.int32, device="cuda")
+    cfg_g = B.config_from_spec(spec, tau=tau, capacity_factor=gamma, flags=B.FLAG_LOGITS_GIVEN)
+    B.moepp_route(cfg_g, lt.x.cuda(), None, None, None, None, None, lg, idx, w, cnt, off, None)
+    ros = torch.empty(spec.T, 2, dtype=torch.int32, device="cuda")
+    sor = torch.empty(cfg.M_cap, dtype=torch.int32, device="cuda")
+    xp = torch.empty(cfg.M_cap, spec.D, dtype=torch.bfloat16, device="cuda")
+    B.moepp_permute(cfg, lt.x.cuda(), idx, off, ros, sor, xp)
+    torch.cuda.synchronize()
+    assert np.array_equal(idx.cpu().numpy(), idx_o)
+    assert np.array_equal(cnt.cpu().numpy(), counts_o) and np.array_equal(off.cpu().numpy(), offsets_o)
+    assert np.array_equal(ros.cpu().numpy(), ros_o) and np.array_equal(sor.cpu().numpy(), sor_o)
+    dropped = (ros_o == -2).mean()
+    assert (dropped == 0) if gamma >= 8 else (dropped > 0.02)
+
+
+def test_balance_stats(oracle64):
+    """Eq. 7 statistics from the router's own outputs."""
+    for spec, tau in ((W.CONFIGS["cfg1_tiny_f32"], 0.75), (W.LayerSpec(T=5000, D=128, F=64, n_ffn=40, n_const=8), 0.1)):
+        lt = W.make_layer(spec, seed=5)
+        cfg = B.config_from_spec(spec, tau=tau)
+        s, oi = shape_of(spec, tau=tau), oracle_inputs(lt)
+        T, N, K = spec.T, spec.N, spec.top_k
+        lg = torch.empty(T, N, device="cuda")
+        idx = torch.empty(T, K, dtype=torch.int32, device="cuda")
+        w = torch.empty(T, K, device="cuda")
+        cnt = torch.empty(N, dtype=torch.int32, device="cuda")
+        off = torch.empty(spec.n_ffn + 1, dtype=torch.int32, device="cuda")
+        B.moepp_route(cfg, lt.x.cuda(), lt.W_r.cuda(), lt.W_g.cuda(), lt.prev.cuda(), None, None, lg, idx, w, cnt, off, None)
+        f = torch.empty(N, device="cuda")
+        P = torch.empty(N, device="cuda")
+        loss = torch.empty(1, device="cuda")
+        B.moepp_balance_stats(cfg, lg, cnt, f, P, loss)
+        torch.cuda.synchronize()
+        f_o, P_o, L_o = oracle64.balance_stats(s, lg.cpu().numpy(), idx.cpu().numpy())
+        assert max_abs(f.cpu().numpy(), f_o) <= 1e-6
+        assert max_abs(P.cpu().numpy(), P_o) <= 1e-6
+        assert abs(float(loss.item()) - L_o) <= 1e-6
+        assert abs(float(f.sum().item()) - K) <= 1e-5
+        # reproducible bit for bit
+        P2 = torch.empty(N, device="cuda")
+        loss2 = torch.empty(1, device="cuda")
+        B.moepp_balance_stats(cfg, lg, cnt, f, P2, loss2)
+        torch.cuda.synchronize()
+        assert torch.equal(P, P2) and torch.equal(loss, loss2)
