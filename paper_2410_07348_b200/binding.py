@@ -207,7 +207,7 @@ def moepp_stack_forward_host(cfg, weights_list, x_host, prev_logits_host, y_host
     _check(lib().moepp_stack_forward_host(ctypes.byref(c), arr, ctypes.c_int32(len(weights_list)), _p(x_host),
                                           _p(prev_logits_host), _p(y_host), _p(logits_out_host), _p(workspace),
                                           ctypes.c_size_t(workspace.numel() * workspace.element_size()), _stream()),
-           "moepp_stack_forward_host", "moepp_balance_stats")
+           "moepp_stack_forward_host")
 
 
 def moepp_device_error() -> int:
