@@ -205,6 +205,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--tokens", type=int, default=0, help="cfg5: token count T")
     ap.add_argument("--zc-share", type=float, default=0.3, help="cfg5: share of slots on zero-computation experts")
+    ap.add_argument("--capacity-factor", type=float, default=0.0, help="Eq. 8 gamma (0 = no capacity limit)")
+    ap.add_argument("--tau", type=float, default=1.0, help="Eq. 7 / Eq. 8 weight of the zero-computation experts")
     ap.add_argument("--layers", type=int, default=0, help="use only the first N layers of the workload (profiling)")
     ap.add_argument("--flags", type=int, default=0, help="MOEPP_FLAG_* bits passed in the configuration")
     args = ap.parse_args()
@@ -236,8 +238,10 @@ def main():
     spec, layers = build_stack(args.workload, W, dev, args.layers, args.tokens, args.zc_share)
     L = len(layers)
     add_res = 1 if L > 1 else 0
-    cfg = B.config_from_spec(spec, add_residual=add_res, flags=args.flags)
-    cfg_v = B.config_from_spec(spec.vanilla(), add_residual=add_res, flags=args.flags)
+    cfg = B.config_from_spec(spec, add_residual=add_res, flags=args.flags, tau=args.tau,
+                             capacity_factor=args.capacity_factor)
+    cfg_v = B.config_from_spec(spec.vanilla(), add_residual=add_res, flags=args.flags, tau=args.tau,
+                               capacity_factor=args.capacity_factor)
     wds = [B.weights_from_tensors(lt, dev) for lt in layers]
     wds_v = [vanilla_weights(wd, spec) for wd in wds]
     x0 = layers[0].x
@@ -310,6 +314,8 @@ def main():
         ("combine", lambda: B.moepp_combine(cfg, x0, yp, idx, wk, ros, alpha if spec.n_const else None, wd["W_c"],
                                             wd["v"], yb)),
     ]
+    f_b, P_b, L_b = torch.empty(N, device=dev), torch.empty(N, device=dev), torch.empty(1, device=dev)
+    calls.append(("balance_stats", lambda: B.moepp_balance_stats(cfg, lgs[0], cnt, f_b, P_b, L_b)))
     reps = max(5, args.steps)
     acc = {n: 0.0 for n, _ in calls}
     for it in range(3 + reps):
@@ -324,6 +330,7 @@ def main():
                 acc[n] += evs[i].elapsed_time(evs[i + 1]) / reps
     counts = cnt.cpu().numpy()
     M = int(off[-1].item())
+    dropped = int((ros == -2).sum().item())
     zc_share = float(counts[spec.n_ffn:].sum()) / float(counts.sum())
     es = 2 if spec.dtype == "bf16" else 4
     flops_ffn = 6.0 * spec.D * spec.F * M
@@ -363,6 +370,8 @@ def main():
         "config": {"workload": key, "layers": L, "T": T, "D": spec.D, "F": spec.F,
                    "experts": "%d+%d" % (spec.n_ffn, spec.n_zc), "top_k": K, "tokens_per_step_per_gpu": tokens_per_step,
                    "zc_slot_share_layer1": round(zc_share, 4), "ffn_rows_layer1": M,
+                   "capacity_factor": args.capacity_factor, "tau": args.tau, "dropped_slots_layer1": dropped,
+                   "balance_loss_layer1": float(L_b.item()),
                    "l2": "inputs larger than L2 (weights %.0f MB per layer); no explicit flush" %
                          (3.0 * spec.D * spec.F * es * spec.n_ffn / 1e6),
                    "parallelism": "replicas: each GPU runs its own token batch, no collective" if world > 1 else "1 GPU"},
