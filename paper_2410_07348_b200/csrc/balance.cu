@@ -7,36 +7,50 @@
 namespace moepp {
 namespace {
 
-constexpr int kBalThreads = 1024;
 
-__global__ void __launch_bounds__(kBalThreads)
+// One thread per token (tokens tid, tid + THREADS, ...), NP >= N per-thread column accumulators in registers
+// (fewer threads for larger NP so that they stay there),
+// then a fixed-order reduction: lanes by shuffle tree, warps in index order.
+template <int NP, int THREADS>
+__global__ void __launch_bounds__(THREADS)
 balance_stats_kernel(Dims dm, const float* __restrict__ logits, const int32_t* __restrict__ counts,
                      float* __restrict__ f, float* __restrict__ P, float* __restrict__ loss) {
-  __shared__ float part[32][kMaxExperts];  // per-warp sums of the softmax columns
-  __shared__ float col[kMaxExperts];
+  __shared__ float part[THREADS / 32][NP];  // per-warp sums of the softmax columns
+  __shared__ float col[NP];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int N = dm.N;
-  // lane i of a warp owns experts i and i + 32; a warp walks tokens warp, warp + 32, ...
-  float acc0 = 0.f, acc1 = 0.f;
-  for (long long t = warp; t < dm.T; t += 32) {
-    const float g0 = (lane < N) ? logits[t * N + lane] : -INFINITY;
-    const float g1 = (lane + 32 < N) ? logits[t * N + lane + 32] : -INFINITY;
-    float m = fmaxf(g0, g1);
+  float acc[NP];
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-    const float p0 = (lane < N) ? expf(g0 - m) : 0.f, p1 = (lane + 32 < N) ? expf(g1 - m) : 0.f;
-    float z = p0 + p1;
+  for (int i = 0; i < NP; ++i) acc[i] = 0.f;
+  for (long long t = tid; t < dm.T; t += THREADS) {
+    const float* row = logits + t * N;
+    float g[NP];
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
-    acc0 += p0 / z;
-    acc1 += p1 / z;
+    for (int i = 0; i < NP; ++i) g[i] = (i < N) ? __ldg(row + i) : -INFINITY;
+    float m = g[0];
+#pragma unroll
+    for (int i = 1; i < NP; ++i) m = fmaxf(m, g[i]);
+    float z = 0.f;
+#pragma unroll
+    for (int i = 0; i < NP; ++i) {
+      g[i] = (i < N) ? expf(g[i] - m) : 0.f;
+      z += g[i];
+    }
+    const float inv = 1.f / z;
+#pragma unroll
+    for (int i = 0; i < NP; ++i) acc[i] = fmaf(g[i], inv, acc[i]);
   }
-  part[warp][lane] = acc0;
-  part[warp][lane + 32] = acc1;
+#pragma unroll
+  for (int i = 0; i < NP; ++i) {
+    float a = acc[i];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+    if (lane == 0) part[warp][i] = a;
+  }
   __syncthreads();
   if (tid < N) {
     float s = 0.f;
-    for (int w = 0; w < 32; ++w) s += part[w][tid];  // fixed order
+    for (int w = 0; w < THREADS / 32; ++w) s += part[w][tid];  // fixed order
     const float inv_T = dm.T > 0 ? 1.f / (float)dm.T : 0.f;
     const float pi = s * inv_T, fi = (float)counts[tid] * inv_T;
     P[tid] = pi;
@@ -55,7 +69,9 @@ balance_stats_kernel(Dims dm, const float* __restrict__ logits, const int32_t* _
 
 cudaError_t launch_balance_stats(const Dims& d, const float* logits, const int32_t* counts, float* f, float* P,
                                  float* loss, cudaStream_t st) {
-  balance_stats_kernel<<<1, kBalThreads, 0, st>>>(d, logits, counts, f, P, loss);
+  if (d.N <= 16) balance_stats_kernel<16, 1024><<<1, 1024, 0, st>>>(d, logits, counts, f, P, loss);
+  else if (d.N <= 32) balance_stats_kernel<32, 512><<<1, 512, 0, st>>>(d, logits, counts, f, P, loss);
+  else balance_stats_kernel<64, 256><<<1, 256, 0, st>>>(d, logits, counts, f, P, loss);
   return cudaGetLastError();
 }
 
