@@ -97,6 +97,7 @@ WORKLOADS = {  # name -> (config key, layers)
     "cfg3": ("cfg3_bf16_16e_skew", 1),
     "cfg2": ("cfg2_bf16_8e", 1),
     "cfg5": ("cfg5_sweep", 1),  # with --tokens and --zc-share
+    "2b": ("paper_2b_32p8e", 1),  # the paper's 2B/(32+8)E layer shape
 }
 
 

@@ -70,6 +70,9 @@ CONFIGS = {
     "cfg3_bf16_16e_skew": LayerSpec(T=32768, D=1536, F=4096, n_ffn=16),
     "cfg4_7b_stack": LayerSpec(T=32768, D=4096, F=2816, n_ffn=16),
     "cfg5_sweep": LayerSpec(T=32768, D=4096, F=2816, n_ffn=16),
+    # the paper's 2B/(32+8)E model (Table 2): hidden 768, intermediate 2048, 32 FFN + 1/1/6 zero-computation
+    # experts; a second router shape (40 experts, 52 stacked rows)
+    "paper_2b_32p8e": LayerSpec(T=32768, D=768, F=2048, n_ffn=32, n_zero=1, n_copy=1, n_const=6),
 }
 CFG4_LAYERS = 4
 CFG5_ZC_SHARES = (0.0, 0.15, 0.30, 0.50, 0.75)

@@ -113,6 +113,14 @@ def test_cfg3_bf16_skewed(oracle64):
     assert c[0] > 8 * c[15]  # Zipf(1.1) over 16 experts: rank 1 carries about 21x rank 16
 
 
+def test_paper_2b_shape_32_plus_8_experts(oracle64):
+    """The paper's 2B/(32+8)E layer (Table 2): 40 experts, six constant experts, 52 stacked router rows."""
+    lt = W.make_config("paper_2b_32p8e", gen_device="cuda", device="cuda")
+    info = check_layer(oracle64, lt, 160)
+    assert 0.1 < info["zc_share"] < 0.35
+    assert np.all(info["counts"] > 0)
+
+
 def test_cfg4_stack_of_four(oracle64):
     """Free-running 4-layer stack on all 32768 tokens; the oracle follows the same picks on a token sample."""
     spec = W.CONFIGS["cfg4_7b_stack"]
