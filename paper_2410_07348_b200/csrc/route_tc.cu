@@ -29,14 +29,14 @@ template <int RP>
 struct RouteTcSmem {
   static constexpr int kBSub = RP * 128;  // one weight term: RP rows of 64 bf16
   static constexpr int kStage = kABytesR + 3 * kBSub;
-  static constexpr int kStages = (RP == 128) ? 2 : 3;  // 128 stacked rows: 64 KiB per stage
+  static constexpr int kStages = (RP == 32) ? 3 : 2;  // 40 / 64 KiB per stage for 64 / 128 stacked rows
   static constexpr int kRing = kStages * kStage;
 };
 
 __device__ __forceinline__ void named_barrier_128() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 template <int RP>
-__global__ void __launch_bounds__(kThreadsR, RP == 32 ? 2 : 1)
+__global__ void __launch_bounds__(kThreadsR, RP <= 64 ? 2 : 1)
 route_tc_kernel(const __grid_constant__ CUtensorMap tmX, Dims dm, const float* __restrict__ W_r,
                 const float* __restrict__ W_g, const float* __restrict__ prev, const float* __restrict__ bias,
                 const float* __restrict__ W_c, float* __restrict__ logits, int32_t* __restrict__ topk_idx,
