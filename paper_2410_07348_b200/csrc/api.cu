@@ -94,8 +94,8 @@ moepp_status ffn_dispatch(const Dims& d, const void* x_perm, const int32_t* offs
   if (d.dtype == MOEPP_BF16 && !(d.flags & MOEPP_FLAG_SIMT_FFN)) {
     const cudaError_t e = ((d.flags & MOEPP_FLAG_FFN_SINGLE_CTA) ? launch_ffn_tcgen05 : launch_ffn_tcgen05_pair)(
         d, x_perm, offsets, W_gate, W_up, W_down, h, y_perm, st);
-    if (e == cudaErrorNotSupported) return MOEPP_ERR_UNSUPPORTED;
-    return from_cuda(e);
+    // a shape the TMA tensor maps cannot describe runs on the FMA kernels instead
+    if (e != cudaErrorNotSupported) return from_cuda(e);
   }
   return from_cuda(launch_ffn_simt(d, x_perm, offsets, W_gate, W_up, W_down, h, y_perm, st));
 }

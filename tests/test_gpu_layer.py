@@ -71,7 +71,8 @@ def check_layer(oracle64, lt, n_sample, host=False, **over):
     idx_o, _ = oracle64.gate_topk(s, r["logits"])
     clear = clear_gap_tokens(r["logits"], spec.top_k)
     assert np.array_equal(idx_g[clear], idx_o[clear])
-    assert clear.mean() > 0.9
+    if spec.T >= 200:
+        assert clear.mean() > 0.9
     got = y.float().cpu().numpy()
     got = got if toks is None else got[toks]
     if spec.dtype == "f32":
@@ -113,6 +114,31 @@ def test_cfg3_bf16_skewed(oracle64):
     assert c[0] > 8 * c[15]  # Zipf(1.1) over 16 experts: rank 1 carries about 21x rank 16
 
 
+@pytest.mark.parametrize("seed", range(8))
+def test_random_shapes(oracle64, seed):
+    """Seeded random small configurations: sizes, expert mix, top-k, padding, capacity, both storage types."""
+    rng = np.random.default_rng(1000 + seed)
+    dtype = "bf16" if seed % 2 == 0 else "f32"
+    n_ffn = int(rng.integers(1, 12))
+    n_zero, n_copy, n_const = int(rng.integers(0, 3)), int(rng.integers(0, 3)), int(rng.integers(0, 4))
+    N = n_ffn + n_zero + n_copy + n_const
+    spec = W.LayerSpec(T=int(rng.integers(1, 1500)), D=8 * int(rng.integers(1, 70)), F=8 * int(rng.integers(1, 70)),
+                       n_ffn=n_ffn, n_zero=n_zero, n_copy=n_copy, n_const=n_const,
+                       top_k=int(rng.integers(1, min(N, 4) + 1)), dtype=dtype)
+    lt = W.make_layer(spec, seed=seed, with_prev=bool(seed & 2), w_std=0.05)
+    over = dict(row_align=int(rng.choice([1, 8, 128])), add_residual=int(rng.integers(0, 2)),
+                renorm_topk=int(rng.integers(0, 2)))
+    if seed % 3 == 0:
+        over.update(capacity_factor=float(rng.choice([0.7, 1.1])), tau=float(rng.choice([0.5, 0.75, 1.0])))
+    check_layer(oracle64, lt, None, **over)
+
+
+def test_tiny_dims_bf16(oracle64):
+    """d_model and d_ffn far below one tile (8 and 16)."""
+    spec = W.LayerSpec(T=300, D=8, F=16, n_ffn=3, dtype="bf16")
+    check_layer(oracle64, W.make_layer(spec, seed=4, w_std=0.3), None)
+
+
 def test_paper_2b_shape_32_plus_8_experts(oracle64):
     """The paper's 2B/(32+8)E layer (Table 2): 40 experts, six constant experts, 52 stacked router rows."""
     lt = W.make_config("paper_2b_32p8e", gen_device="cuda", device="cuda")
@@ -135,12 +161,14 @@ def test_cfg4_stack_of_four(oracle64):
     x_o = None
     prev_o = None
     s_sub = shape_of(sub, add_residual=1)
+    kept, x_first = [], None
     for j in range(1, 5):
         # build one layer at a time to bound memory: same recipe as workloads.make_stack
         lt = W.make_layer(spec if j == 1 else W.LayerSpec(0, spec.D, spec.F, spec.n_ffn, dtype="bf16"), seed=j - 1,
                           with_prev=False, w_std=0.02 / math.sqrt(j), device="cuda", gen_device="cuda")
         if j == 1:
             x = lt.x
+            x_first = x
             x_o = f32(x)[toks]
         else:
             g = torch.Generator(device="cuda").manual_seed(1000 + j)
@@ -174,7 +202,16 @@ def test_cfg4_stack_of_four(oracle64):
         assert np.array_equal(idx_g[clear], idx_o[clear])
         x, prev = y, logits
         x_o, prev_o = r["y"], r["logits"]
-        del lt, wd
+        kept.append(wd)
+        del lt
+    # the call bench.py times: the whole stack in one moepp_stack_forward, same bits as the chained calls
+    ws2 = torch.empty(B.moepp_stack_workspace_bytes(cfg, 4), dtype=torch.uint8, device="cuda")
+    y2 = torch.empty_like(x)
+    lg2 = torch.empty(spec.T, spec.N, device="cuda")
+    B.moepp_stack_forward(cfg, kept, x_first, None, y2, lg2, ws2)
+    torch.cuda.synchronize()
+    assert B.moepp_device_error() == 0
+    assert torch.equal(y2, x) and torch.equal(lg2, prev)
 
 
 def test_stack_call_equals_chained_layer_calls(oracle64):
