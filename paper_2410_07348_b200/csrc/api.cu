@@ -368,14 +368,57 @@ moepp_status moepp_stack_forward(const moepp_config* cfg, const moepp_weights* l
                          static_cast<cudaStream_t>(stream));
 }
 
+// ---- stack with host activations: token chunks pipelined over copy-in, compute and copy-out ----------------
+// Tokens are independent through a stack (no capacity limit), so the batch is cut into chunks: while one chunk
+// computes on the caller's stream, the next one is copied in and the previous one copied out on two internal
+// streams.  Every chunk owns its own slice of the workspace.
+namespace {
+
+struct HostChunks {
+  int n;        // number of chunks
+  int tokens;   // tokens per chunk (a multiple of 128; the last chunk takes the rest)
+};
+
+HostChunks host_chunks(const Dims& d) {
+  HostChunks h{1, d.T};
+  if (d.cap_on) return h;  // Eq. 8 shares one capacity among all tokens: keep the batch whole
+  const int n = d.T >= 16384 ? 4 : (d.T >= 4096 ? 2 : 1);
+  if (n > 1) {
+    h.n = n;
+    h.tokens = ((d.T + n - 1) / n + 127) / 128 * 128;
+    h.n = (d.T + h.tokens - 1) / h.tokens;
+  }
+  return h;
+}
+
+Dims chunk_dims(const Dims& d, int tokens) {
+  Dims c = d;
+  c.T = tokens;
+  c.M_cap = (long long)tokens * d.K + (long long)d.n_ffn * (d.row_align - 1);
+  return c;
+}
+
+// workspace of one chunk: layer workspace + ping-pong buffers + staging of x, y, prev, last logits
+size_t chunk_ws_bytes(const Dims& c) {
+  size_t act, lg;
+  const size_t extra = stack_extra_bytes(c, &act, &lg);
+  return carve(c, false).total + extra + 2 * act + 2 * lg;
+}
+
+}  // namespace
+
 moepp_status moepp_stack_workspace_bytes_host(const moepp_config* cfg, int32_t n_layers, size_t* bytes) {
   Dims d;
   const moepp_status s = make_dims(cfg, &d);
   if (s != MOEPP_OK) return s;
   if (bytes == nullptr || n_layers < 1) return MOEPP_ERR_INVALID_ARG;
-  size_t act, lg;
-  const size_t extra = stack_extra_bytes(d, &act, &lg);
-  *bytes = carve(d, false).total + extra + 2 * act + 2 * lg;  // + staging of x, y, prev and the last logits
+  const HostChunks h = host_chunks(d);
+  size_t total = 0;
+  for (int i = 0; i < h.n; ++i) {
+    const int tok = (i + 1 < h.n) ? h.tokens : d.T - i * h.tokens;
+    total += chunk_ws_bytes(chunk_dims(d, tok));
+  }
+  *bytes = total;
   return MOEPP_OK;
 }
 
@@ -388,33 +431,96 @@ moepp_status moepp_stack_forward_host(const moepp_config* cfg, const moepp_weigh
   if (layers == nullptr || n_layers < 1 || workspace == nullptr) return MOEPP_ERR_INVALID_ARG;
   if (d.T > 0 && (x_host == nullptr || y_host == nullptr)) return MOEPP_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) != 0) return MOEPP_ERR_ALIGN;
-  size_t act, lg;
-  const size_t extra = stack_extra_bytes(d, &act, &lg);
-  const size_t base = carve(d, false).total + extra;
-  if (workspace_bytes < base + 2 * act + 2 * lg) return MOEPP_ERR_WORKSPACE;
+  size_t need = 0;
+  {
+    const moepp_status w = moepp_stack_workspace_bytes_host(cfg, n_layers, &need);
+    if (w != MOEPP_OK) return w;
+  }
+  if (workspace_bytes < need) return MOEPP_ERR_WORKSPACE;
   if (d.T > 0 && layers[0].W_g != nullptr && prev_logits_host == nullptr) return MOEPP_ERR_INVALID_ARG;
   if (d.T == 0) return MOEPP_OK;
-  char* ws = static_cast<char*>(workspace);
+
+  const HostChunks h = host_chunks(d);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  char* x_dev = ws + base;
-  char* y_dev = x_dev + act;
-  float* p_dev = reinterpret_cast<float*>(y_dev + act);
-  float* l_dev = reinterpret_cast<float*>(y_dev + act + lg);
-  const size_t act_bytes = elem_size(d.dtype) * (size_t)d.T * d.D, lg_bytes = sizeof(float) * (size_t)d.T * d.N;
-  if (cudaMemcpyAsync(x_dev, x_host, act_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return MOEPP_ERR_CUDA;
-  const float* prev = nullptr;
-  if (prev_logits_host != nullptr) {
-    if (cudaMemcpyAsync(p_dev, prev_logits_host, lg_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
-      return MOEPP_ERR_CUDA;
-    prev = p_dev;
+  const size_t es = elem_size(d.dtype);
+  constexpr int kMaxChunks = 8;
+  cudaStream_t s_in = nullptr, s_out = nullptr;
+  cudaEvent_t ev_start = nullptr, ev_out = nullptr, ev_in[kMaxChunks] = {}, ev_done[kMaxChunks] = {};
+  const bool piped = h.n > 1;
+  moepp_status result = MOEPP_OK;
+  auto fail = [&](moepp_status code) { if (result == MOEPP_OK) result = code; };
+
+  if (piped) {  // two internal streams and a handful of events, created and released inside this call
+    bool ok = cudaStreamCreateWithFlags(&s_in, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&s_out, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&ev_start, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&ev_out, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; ok && i < h.n; ++i)
+      ok = cudaEventCreateWithFlags(&ev_in[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&ev_done[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) fail(MOEPP_ERR_CUDA);
+    // the internal streams start after whatever the caller queued before this call
+    if (result == MOEPP_OK && (cudaEventRecord(ev_start, st) != cudaSuccess ||
+                               cudaStreamWaitEvent(s_in, ev_start, 0) != cudaSuccess ||
+                               cudaStreamWaitEvent(s_out, ev_start, 0) != cudaSuccess))
+      fail(MOEPP_ERR_CUDA);
   }
-  const moepp_status r = stack_on_device(d, layers, n_layers, x_dev, prev, y_dev, l_dev, ws, st);
-  if (r != MOEPP_OK) return r;
-  if (cudaMemcpyAsync(y_host, y_dev, act_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return MOEPP_ERR_CUDA;
-  if (logits_out_host != nullptr &&
-      cudaMemcpyAsync(logits_out_host, l_dev, lg_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
-    return MOEPP_ERR_CUDA;
-  return MOEPP_OK;
+
+  char* ws = static_cast<char*>(workspace);
+  for (int i = 0; i < h.n && result == MOEPP_OK; ++i) {
+    const int t_begin = i * h.tokens;
+    const int tok = (i + 1 < h.n) ? h.tokens : d.T - t_begin;
+    const Dims c = chunk_dims(d, tok);
+    size_t act, lg;
+    const size_t extra = stack_extra_bytes(c, &act, &lg);
+    const size_t base = carve(c, false).total + extra;
+    char* x_dev = ws + base;
+    char* y_dev = x_dev + act;
+    float* p_dev = reinterpret_cast<float*>(y_dev + act);
+    float* l_dev = reinterpret_cast<float*>(y_dev + act + lg);
+    const size_t act_bytes = es * (size_t)tok * d.D, lg_bytes = sizeof(float) * (size_t)tok * d.N;
+    const char* xh = static_cast<const char*>(x_host) + es * (size_t)t_begin * d.D;
+    char* yh = static_cast<char*>(y_host) + es * (size_t)t_begin * d.D;
+    cudaStream_t cin = piped ? s_in : st, cout = piped ? s_out : st;
+
+    if (cudaMemcpyAsync(x_dev, xh, act_bytes, cudaMemcpyHostToDevice, cin) != cudaSuccess) { fail(MOEPP_ERR_CUDA); break; }
+    const float* prev = nullptr;
+    if (prev_logits_host != nullptr) {
+      if (cudaMemcpyAsync(p_dev, prev_logits_host + (size_t)t_begin * d.N, lg_bytes, cudaMemcpyHostToDevice, cin) !=
+          cudaSuccess) { fail(MOEPP_ERR_CUDA); break; }
+      prev = p_dev;
+    }
+    if (piped && (cudaEventRecord(ev_in[i], s_in) != cudaSuccess || cudaStreamWaitEvent(st, ev_in[i], 0) != cudaSuccess)) {
+      fail(MOEPP_ERR_CUDA); break;
+    }
+    const moepp_status r = stack_on_device(c, layers, n_layers, x_dev, prev, y_dev, l_dev, ws, st);
+    if (r != MOEPP_OK) { fail(r); break; }
+    if (piped && (cudaEventRecord(ev_done[i], st) != cudaSuccess ||
+                  cudaStreamWaitEvent(s_out, ev_done[i], 0) != cudaSuccess)) { fail(MOEPP_ERR_CUDA); break; }
+    if (cudaMemcpyAsync(yh, y_dev, act_bytes, cudaMemcpyDeviceToHost, cout) != cudaSuccess) { fail(MOEPP_ERR_CUDA); break; }
+    if (logits_out_host != nullptr &&
+        cudaMemcpyAsync(logits_out_host + (size_t)t_begin * d.N, l_dev, lg_bytes, cudaMemcpyDeviceToHost, cout) !=
+            cudaSuccess) { fail(MOEPP_ERR_CUDA); break; }
+    ws += chunk_ws_bytes(c);
+  }
+
+  if (piped) {
+    // the caller's stream ends after the last copy out; then the internal objects go (the runtime frees them
+    // once the work queued on them has finished)
+    if (s_out != nullptr && ev_out != nullptr) {
+      if (cudaEventRecord(ev_out, s_out) != cudaSuccess || cudaStreamWaitEvent(st, ev_out, 0) != cudaSuccess)
+        fail(MOEPP_ERR_CUDA);
+    }
+    for (int i = 0; i < h.n; ++i) {
+      if (ev_in[i]) cudaEventDestroy(ev_in[i]);
+      if (ev_done[i]) cudaEventDestroy(ev_done[i]);
+    }
+    if (ev_start) cudaEventDestroy(ev_start);
+    if (ev_out) cudaEventDestroy(ev_out);
+    if (s_in) cudaStreamDestroy(s_in);
+    if (s_out) cudaStreamDestroy(s_out);
+  }
+  return result;
 }
 
 moepp_status moepp_balance_stats(const moepp_config* cfg, const float* logits, const int32_t* expert_counts, float* f,

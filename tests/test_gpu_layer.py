@@ -262,6 +262,30 @@ def test_stack_call_equals_chained_layer_calls(oracle64):
         cur, prev, x_o, prev_o = y, lg, r["y"], r["logits"]
 
 
+@pytest.mark.parametrize("T", [5000, 20000])
+def test_host_stack_call_chunks_tokens(T):
+    """The host-buffer stack call cuts large batches into token chunks that overlap copies with compute; the
+    result must be the same bits as the device call on the whole batch."""
+    spec = W.LayerSpec(T=T, D=256, F=384, n_ffn=6, dtype="bf16")
+    layers = W.make_stack(spec, 2, device="cuda", gen_device="cuda")
+    cfg = B.config_from_spec(spec, add_residual=1)
+    wds = [B.weights_from_tensors(lt) for lt in layers]
+    x = layers[0].x
+    ws = torch.empty(B.moepp_stack_workspace_bytes(cfg, 2), dtype=torch.uint8, device="cuda")
+    y = torch.empty_like(x)
+    lg = torch.empty(T, spec.N, device="cuda")
+    B.moepp_stack_forward(cfg, wds, x, None, y, lg, ws)
+    wsh = torch.empty(B.moepp_stack_workspace_bytes(cfg, 2, host=True), dtype=torch.uint8, device="cuda")
+    xh = x.cpu().pin_memory()
+    for _ in range(2):  # twice in a row: the second call must wait for nothing it should not and reuse cleanly
+        yh = torch.zeros_like(x, device="cpu").pin_memory()
+        lh = torch.zeros(T, spec.N).pin_memory()
+        B.moepp_stack_forward_host(cfg, wds, xh, None, yh, lh, wsh)
+        torch.cuda.current_stream().synchronize()
+        assert torch.equal(yh, y.cpu()) and torch.equal(lh, lg.cpu())
+    assert B.moepp_device_error() == 0
+
+
 def test_cfg4_teacher_forced_layers(oracle64):
     """Each layer of the stack fed the oracle's own state (rounded once to bf16): picks exact, outputs in tolerance."""
     spec = W.CONFIGS["cfg4_7b_stack"]
