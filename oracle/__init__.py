@@ -207,3 +207,20 @@ class Oracle:
                    _ptr(W_c), _ptr(v), _ptr(W_gate), _ptr(W_up), _ptr(W_down), _ptr(forced_idx), _ptr(tokens),
                    ctypes.c_int32(0 if tokens is None else len(tokens)), _ptr(logits), _ptr(idx), _ptr(w), _ptr(y))
         return dict(logits=logits, idx=idx, w=w, y=y)
+
+    def layer_backward(self, s, x, W_r, idx, dy, W_g=None, prev=None, bias=None, W_c=None, v=None, W_gate=None,
+                       W_up=None, W_down=None, dlogits=None):
+        """Gradients of a scalar L given dy = dL/dy (and dlogits = dL/dlogits from the next layer), with the picks
+        `idx` held fixed.  Returns a dict with dx, dprev, dW_r, dW_g, dbias, dW_c, dv, dW_gate, dW_up, dW_down."""
+        x, W_r, W_g, prev, bias, W_c, v = _f32(x), _f32(W_r), _f32(W_g), _f32(prev), _f32(bias), _f32(W_c), _f32(v)
+        W_gate, W_up, W_down, dy, dlogits, idx = _f32(W_gate), _f32(W_up), _f32(W_down), _f32(dy), _f32(dlogits), _i32(idx)
+        z = lambda *shape: np.zeros(shape, np.float32)
+        out = dict(dx=z(s.T, s.D), dprev=z(s.T, s.N) if W_g is not None else None, dW_r=z(s.N, s.D),
+                   dW_g=z(s.N, s.N) if W_g is not None else None, dbias=z(s.N), dW_c=z(max(s.n_const, 0), 2, s.D),
+                   dv=z(max(s.n_const, 0), s.D), dW_gate=z(s.n_ffn, s.F, s.D), dW_up=z(s.n_ffn, s.F, s.D),
+                   dW_down=z(s.n_ffn, s.D, s.F))
+        self._call("layer_backward", self._cfg(s), _ptr(x), _ptr(W_r), _ptr(W_g), _ptr(prev), _ptr(bias), _ptr(W_c),
+                   _ptr(v), _ptr(W_gate), _ptr(W_up), _ptr(W_down), _ptr(idx), _ptr(dy), _ptr(dlogits),
+                   _ptr(out["dx"]), _ptr(out["dprev"]), _ptr(out["dW_r"]), _ptr(out["dW_g"]), _ptr(out["dbias"]),
+                   _ptr(out["dW_c"]), _ptr(out["dv"]), _ptr(out["dW_gate"]), _ptr(out["dW_up"]), _ptr(out["dW_down"]))
+        return out

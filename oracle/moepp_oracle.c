@@ -445,3 +445,194 @@ int FN(balance_stats)(const oracle_config* c, const float* G, const int32_t* idx
   *loss = (float)L;
   return 0;
 }
+
+/* ==== backward pass: chain rule through Eq. 1-6, token by token ===================================== */
+
+/* gradient accumulators for the weights, in `real`, rounded to float once at the end */
+static real* zeros_real(size_t n) { return (real*)calloc(n > 0 ? n : 1, sizeof(real)); }
+static void store_f32(float* dst, const real* src, size_t n) {
+  if (!dst) return;
+  for (size_t i = 0; i < n; ++i) dst[i] = (float)src[i];
+}
+
+/* one FFN expert on token u: forward values kept, then the gradient of dc = dL/d(out) */
+static void ffn_backward_token(const oracle_config* c, const real* u, const float* Wg, const float* Wu,
+                               const float* Wd, const real* dc, real* du, real* gWg, real* gWu, real* gWd,
+                               real* out, real* scratch) {
+  const int D = c->D, F = c->F;
+  real *gt = scratch, *up = scratch + F, *sg = scratch + 2 * F, *h = scratch + 3 * F, *dh = scratch + 4 * F;
+  for (int f = 0; f < F; ++f) {
+    real a = 0, b = 0;
+    for (int d = 0; d < D; ++d) {
+      a += (real)Wg[(int64_t)f * D + d] * u[d];
+      b += (real)Wu[(int64_t)f * D + d] * u[d];
+    }
+    gt[f] = a;
+    up[f] = b;
+    sg[f] = (real)1 / ((real)1 + r_exp(-a)); /* sigmoid */
+    h[f] = a * sg[f] * b;                     /* silu(gate) * up */
+  }
+  for (int d = 0; d < D; ++d) {
+    real o = 0;
+    for (int f = 0; f < F; ++f) o += (real)Wd[(int64_t)d * F + f] * h[f];
+    out[d] = o;
+  }
+  if (!dc) return;
+  for (int f = 0; f < F; ++f) {
+    real a = 0;
+    for (int d = 0; d < D; ++d) a += dc[d] * (real)Wd[(int64_t)d * F + f];
+    dh[f] = a;
+  }
+  for (int d = 0; d < D; ++d)
+    for (int f = 0; f < F; ++f) gWd[(int64_t)d * F + f] += dc[d] * h[f];
+  for (int f = 0; f < F; ++f) {
+    const real d_up = dh[f] * gt[f] * sg[f];
+    /* d silu(z)/dz = s + z s (1 - s) */
+    const real d_gt = dh[f] * up[f] * (sg[f] + gt[f] * sg[f] * ((real)1 - sg[f]));
+    for (int d = 0; d < D; ++d) {
+      gWg[(int64_t)f * D + d] += d_gt * u[d];
+      gWu[(int64_t)f * D + d] += d_up * u[d];
+      du[d] += d_gt * (real)Wg[(int64_t)f * D + d] + d_up * (real)Wu[(int64_t)f * D + d];
+    }
+  }
+}
+
+int FN(layer_backward)(const oracle_config* c, const float* x, const float* W_r, const float* W_g, const float* prev,
+                       const float* bias, const float* W_c, const float* v, const float* W_gate, const float* W_up,
+                       const float* W_down, const int32_t* idx, const float* dy, const float* dlogits, float* dx,
+                       float* dprev, float* dW_r, float* dW_g, float* dbias, float* dW_c, float* dv, float* dW_gate,
+                       float* dW_up, float* dW_down) {
+  if (bad_config(c) || !x || !W_r || !idx || !dy || !dx || !dW_r) return 1;
+  if ((W_g == NULL) != (prev == NULL)) return 1;
+  const int N = n_experts(c), D = c->D, F = c->F, K = c->top_k, T = c->T;
+  if (N > 256 || c->ffn_w_bf16) return 1;
+  const int zero0 = c->n_ffn, copy0 = zero0 + c->n_zero, const0 = copy0 + c->n_copy;
+  const int64_t DF = (int64_t)D * F;
+
+  real* gWr = zeros_real((size_t)N * D);
+  real* gWgate = zeros_real((size_t)c->n_ffn * DF), *gWup = zeros_real((size_t)c->n_ffn * DF);
+  real* gWdown = zeros_real((size_t)c->n_ffn * DF);
+  real* gWg = zeros_real((size_t)N * N), *gb = zeros_real((size_t)N);
+  real* gWc = zeros_real((size_t)c->n_const * 2 * D), *gv = zeros_real((size_t)c->n_const * D);
+  real* buf = (real*)malloc(sizeof(real) * (size_t)(4 * D + 5 * F + 8));
+  real *u = buf, *du = buf + D, *dc = buf + 2 * D, *out = buf + 3 * D, *scratch = buf + 4 * D;
+
+  /* Eq. 8: which slots were dropped (same rule as the forward pass) */
+  int32_t cap_ffn, cap_zc;
+  oracle_capacities(c, &cap_ffn, &cap_zc);
+  char* dropped = (char*)calloc((size_t)T * K + 1, 1);
+  if (c->capacity_factor > 0.0f) {
+    int32_t seen[256];
+    memset(seen, 0, sizeof seen);
+    for (int64_t s = 0; s < (int64_t)T * K; ++s) {
+      const int e = idx[s];
+      if (seen[e] >= (e < zero0 ? cap_ffn : cap_zc)) dropped[s] = 1;
+      seen[e] += 1;
+    }
+  }
+
+  for (int t = 0; t < T; ++t) {
+    const float* xt = x + (int64_t)t * D;
+    const float* dyt = dy + (int64_t)t * D;
+    real g[256], P[256], wk[256], dw[256], dG[256];
+    logits_token(c, xt, W_r, W_g, prev ? prev + (int64_t)t * N : NULL, bias, g);
+    for (int i = 0; i < N; ++i) g[i] = (real)(float)g[i]; /* the forward pass stores the logits in float */
+    softmax_all(g, N, P);
+    real S = 0;
+    for (int k = 0; k < K; ++k) S += P[idx[(int64_t)t * K + k]];
+    for (int k = 0; k < K; ++k) {
+      wk[k] = P[idx[(int64_t)t * K + k]];
+      if (c->renorm_topk) wk[k] = wk[k] / S;
+      wk[k] = (real)(float)wk[k]; /* stored in float by the forward pass */
+    }
+    for (int d = 0; d < D; ++d) {
+      u[d] = (real)xt[d];
+      du[d] = c->add_residual ? (real)dyt[d] : (real)0; /* y = x + ... */
+    }
+    for (int k = 0; k < K; ++k) {
+      const int e = idx[(int64_t)t * K + k];
+      dw[k] = 0;
+      if (dropped[(int64_t)t * K + k]) continue;
+      for (int d = 0; d < D; ++d) dc[d] = wk[k] * (real)dyt[d]; /* dL/d E_k(x) */
+      if (e < zero0) {
+        ffn_backward_token(c, u, W_gate + e * DF, W_up + e * DF, W_down + e * DF, dc, du, gWgate + e * DF,
+                           gWup + e * DF, gWdown + e * DF, out, scratch);
+        for (int d = 0; d < D; ++d) dw[k] += (real)dyt[d] * out[d];
+      } else if (e < copy0) {
+        /* Eq. 3: E = 0, nothing flows */
+      } else if (e < const0) { /* Eq. 4: E = x */
+        for (int d = 0; d < D; ++d) {
+          dw[k] += (real)dyt[d] * u[d];
+          du[d] += dc[d];
+        }
+      } else { /* Eq. 5: E = a1 x + a2 v, a = softmax(W_c x) */
+        const int q = e - const0;
+        const float* Wc = W_c + (int64_t)q * 2 * D;
+        const float* vq = v + (int64_t)q * D;
+        real a[2];
+        alpha_token(c, xt, Wc, a);
+        real da1 = 0, da2 = 0;
+        for (int d = 0; d < D; ++d) {
+          dw[k] += (real)dyt[d] * (a[0] * u[d] + a[1] * (real)vq[d]);
+          da1 += dc[d] * u[d];
+          da2 += dc[d] * (real)vq[d];
+          du[d] += a[0] * dc[d];
+          gv[(int64_t)q * D + d] += a[1] * dc[d];
+        }
+        const real mean = a[0] * da1 + a[1] * da2; /* softmax backward over the two mixing logits */
+        const real dz0 = a[0] * (da1 - mean), dz1 = a[1] * (da2 - mean);
+        for (int d = 0; d < D; ++d) {
+          gWc[((int64_t)q * 2 + 0) * D + d] += dz0 * u[d];
+          gWc[((int64_t)q * 2 + 1) * D + d] += dz1 * u[d];
+          du[d] += dz0 * (real)Wc[d] + dz1 * (real)Wc[D + d];
+        }
+      }
+    }
+    /* gate: w_k = P[idx_k] (/ sum over the picks if renormalised); softmax over all N */
+    real dP[256];
+    for (int i = 0; i < N; ++i) dP[i] = 0;
+    if (c->renorm_topk) {
+      real dot = 0;
+      for (int k = 0; k < K; ++k) dot += dw[k] * wk[k];
+      for (int k = 0; k < K; ++k) dP[idx[(int64_t)t * K + k]] += (dw[k] - dot) / S;
+    } else {
+      for (int k = 0; k < K; ++k) dP[idx[(int64_t)t * K + k]] += dw[k];
+    }
+    real dotP = 0;
+    for (int i = 0; i < N; ++i) dotP += dP[i] * P[i];
+    for (int i = 0; i < N; ++i) {
+      dG[i] = P[i] * (dP[i] - dotP);
+      if (dlogits) dG[i] += (real)dlogits[(int64_t)t * N + i]; /* the next layer's gating residual reads G */
+    }
+    /* router: G = W_r x + W_g G_prev + b */
+    for (int i = 0; i < N; ++i) {
+      for (int d = 0; d < D; ++d) {
+        gWr[(int64_t)i * D + d] += dG[i] * u[d];
+        du[d] += dG[i] * (real)W_r[(int64_t)i * D + d];
+      }
+      gb[i] += dG[i];
+    }
+    if (W_g) {
+      for (int j = 0; j < N; ++j) {
+        real a = 0;
+        for (int i = 0; i < N; ++i) {
+          a += dG[i] * (real)W_g[i * N + j];
+          gWg[i * N + j] += dG[i] * (real)prev[(int64_t)t * N + j];
+        }
+        if (dprev) dprev[(int64_t)t * N + j] = (float)a;
+      }
+    }
+    for (int d = 0; d < D; ++d) dx[(int64_t)t * D + d] = (float)du[d];
+  }
+  store_f32(dW_r, gWr, (size_t)N * D);
+  store_f32(dW_g, gWg, (size_t)N * N);
+  store_f32(dbias, gb, (size_t)N);
+  store_f32(dW_c, gWc, (size_t)c->n_const * 2 * D);
+  store_f32(dv, gv, (size_t)c->n_const * D);
+  store_f32(dW_gate, gWgate, (size_t)c->n_ffn * DF);
+  store_f32(dW_up, gWup, (size_t)c->n_ffn * DF);
+  store_f32(dW_down, gWdown, (size_t)c->n_ffn * DF);
+  free(gWr); free(gWgate); free(gWup); free(gWdown); free(gWg); free(gb); free(gWc); free(gv); free(buf);
+  free(dropped);
+  return 0;
+}

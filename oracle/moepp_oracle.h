@@ -104,8 +104,24 @@ int oracle_num_threads(void);
                        const int32_t* forced_idx, const int32_t* tokens, int32_t n_tokens,         \
                        float* logits, int32_t* idx, float* w, float* y);
 
+/* Backward pass of the layer: the gradient of a scalar L with respect to every input, given
+ * dy = dL/dy [T,D] and (may be NULL) dlogits = dL/dlogits [T,N] arriving from the next layer's
+ * gating residual (Eq. 6).  It is the chain rule written out token by token for Eq. 1-6 with the picks
+ * `idx` held fixed (top-K itself has no gradient; slots dropped by Eq. 8 have none either).
+ * All gradient outputs are float arrays of the shape of the thing they belong to; dprev, dW_g, dbias may be
+ * NULL when the layer has no such input.  FFN weights must be float here. */
+#define ORACLE_DECLARE_BWD(P)                                                                          \
+  int P##layer_backward(const oracle_config* c, const float* x, const float* W_r, const float* W_g,    \
+                        const float* prev, const float* bias, const float* W_c, const float* v,        \
+                        const float* W_gate, const float* W_up, const float* W_down,                   \
+                        const int32_t* idx, const float* dy, const float* dlogits, float* dx,          \
+                        float* dprev, float* dW_r, float* dW_g, float* dbias, float* dW_c, float* dv,  \
+                        float* dW_gate, float* dW_up, float* dW_down);
+
 ORACLE_DECLARE(oracle_f32_)
 ORACLE_DECLARE(oracle_f64_)
+ORACLE_DECLARE_BWD(oracle_f32_)
+ORACLE_DECLARE_BWD(oracle_f64_)
 
 #ifdef __cplusplus
 }
