@@ -213,6 +213,51 @@ moepp_status moepp_stack_forward_host(const moepp_config* cfg, const moepp_weigh
                                       float* logits_out_host, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Backward pass of one layer: the chain rule through Eq. 1-6 with the top-K picks held fixed (the
+ * selection is piecewise constant).  The paper trains the layer with ordinary back-propagation and
+ * prints no formulas for it; these are the derivatives of the forward pass above.
+ *
+ * Every pointer of moepp_grads is device memory the caller owns; every gradient is OVERWRITTEN
+ * (not accumulated).  Weight gradients are float whatever cfg->dtype is; dx has cfg->dtype.
+ */
+typedef struct {
+  void* dx;       /* [T, D]  dL/dx, cfg->dtype */
+  float* dprev;   /* [T, N]  dL/dprev_logits; required when weights->W_g is set, else ignored */
+  float* dW_r;    /* [N, D] */
+  float* dW_g;    /* [N, N]  may be NULL */
+  float* dbias;   /* [N]     may be NULL */
+  float* dW_c;    /* [n_const, 2, D]  required when n_const > 0 */
+  float* dv;      /* [n_const, D]     required when n_const > 0 */
+  float* dW_gate; /* [n_ffn, F, D]    required when n_ffn > 0 */
+  float* dW_up;   /* [n_ffn, F, D] */
+  float* dW_down; /* [n_ffn, D, F] */
+} moepp_grads;
+
+/* Bytes of device scratch moepp_layer_backward needs on top of the forward workspace. */
+moepp_status moepp_backward_workspace_bytes(const moepp_config* cfg, size_t* bytes);
+
+/*
+ * Device pointers.  `fwd_workspace` is the workspace moepp_layer_forward filled for the SAME cfg, weights,
+ * x and prev_logits (it holds the picks, gate weights, row tables, grouped activations and the SwiGLU
+ * output); it is read, not written.  `logits` is what that forward call returned in logits_out, or NULL
+ * if logits_out was NULL there (the copy in the workspace is used).
+ *   dy           [T, D] cfg->dtype   dL/dy
+ *   dlogits_next [T, N] float or NULL: dL/dlogits arriving from the next layer's gating residual (Eq. 6)
+ * Steps: combine backward (dL/dE_k = w_k dy to the grouped rows, dL/dw_k = <dy, E_k(x)>; Eq. 3 passes
+ * nothing, Eq. 4 passes w dy to x, Eq. 5 also feeds dv and the two mixing logits), gate backward (softmax
+ * over all N, renormalisation if on), the expert FFNs (SwiGLU pre-activations recomputed from x_perm),
+ * the router (dW_r, dW_g, dbias, dprev) and dx.  Slots dropped by Eq. 8 carry no gradient.
+ * The FFN GEMMs of this pass run on the FMA units (float accumulation) for both dtypes.
+ * MOEPP_FLAG_FUSED_GATHER is refused (that forward path does not keep x_perm).
+ * Errors: as moepp_layer_forward; MOEPP_ERR_WORKSPACE when either workspace is too small.
+ */
+moepp_status moepp_layer_backward(const moepp_config* cfg, const moepp_weights* weights, const void* x,
+                                  const float* prev_logits, const float* logits, const void* dy,
+                                  const float* dlogits_next, const void* fwd_workspace, size_t fwd_workspace_bytes,
+                                  const moepp_grads* grads, void* bwd_workspace, size_t bwd_workspace_bytes,
+                                  void* stream);
+
+/*
  * moepp_grouped_ffn without a scratch argument.  (The paper has no counterpart to this call: it exists
  * for the way this library is embedded, not for the method.)
  *

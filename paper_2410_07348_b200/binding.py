@@ -25,7 +25,8 @@ EXPORTS = ("moepp_status_string", "moepp_workspace_bytes", "moepp_workspace_byte
            "moepp_permute", "moepp_grouped_ffn", "moepp_combine", "moepp_layer_forward",
            "moepp_layer_forward_host", "moepp_device_error", "moepp_grouped_ffn_static",
            "moepp_stack_workspace_bytes", "moepp_stack_forward", "moepp_stack_workspace_bytes_host",
-           "moepp_stack_forward_host", "moepp_balance_stats")
+           "moepp_stack_forward_host", "moepp_balance_stats", "moepp_backward_workspace_bytes",
+           "moepp_layer_backward")
 STATIC_SCRATCH_BYTES = 32 << 20
 
 
@@ -43,6 +44,11 @@ class moepp_config(ctypes.Structure):
 
 class moepp_weights(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in ("W_r", "W_g", "W_c", "v", "router_bias", "W_gate", "W_up", "W_down")]
+
+
+class moepp_grads(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("dx", "dprev", "dW_r", "dW_g", "dbias", "dW_c", "dv", "dW_gate",
+                                               "dW_up", "dW_down")]
 
 
 def lib() -> ctypes.CDLL:
@@ -170,6 +176,26 @@ def moepp_layer_forward_host(cfg, weights: dict, x_host, prev_logits_host, y_hos
                                           _p(y_host), _p(logits_out_host), _p(workspace),
                                           ctypes.c_size_t(workspace.numel() * workspace.element_size()), _stream()),
            "moepp_layer_forward_host")
+
+
+def moepp_backward_workspace_bytes(cfg: Config) -> int:
+    n = ctypes.c_size_t(0)
+    c = cfg.c()
+    _check(lib().moepp_backward_workspace_bytes(ctypes.byref(c), ctypes.byref(n)), "moepp_backward_workspace_bytes")
+    return int(n.value)
+
+
+def moepp_layer_backward(cfg, weights: dict, x, prev_logits, logits, dy, dlogits_next, fwd_workspace, grads: dict,
+                         bwd_workspace):
+    """grads: dict of CUDA tensors named like the fields of moepp_grads (absent or None = NULL)."""
+    c, w = cfg.c(), _weights(weights)
+    g = moepp_grads()
+    for name, _ in moepp_grads._fields_:
+        setattr(g, name, _p(grads.get(name)))
+    nbytes = lambda t: ctypes.c_size_t(t.numel() * t.element_size())
+    _check(lib().moepp_layer_backward(ctypes.byref(c), ctypes.byref(w), _p(x), _p(prev_logits), _p(logits), _p(dy),
+                                      _p(dlogits_next), _p(fwd_workspace), nbytes(fwd_workspace), ctypes.byref(g),
+                                      _p(bwd_workspace), nbytes(bwd_workspace), _stream()), "moepp_layer_backward")
 
 
 def moepp_balance_stats(cfg, logits, expert_counts, f, P, loss):

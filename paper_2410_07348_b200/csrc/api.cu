@@ -533,6 +533,91 @@ moepp_status moepp_balance_stats(const moepp_config* cfg, const float* logits, c
   return from_cuda(launch_balance_stats(d, logits, expert_counts, f, P, loss, static_cast<cudaStream_t>(stream)));
 }
 
+// Device scratch of the backward pass, carved like the forward workspace.
+struct BwdCarve {
+  size_t dYp, gate, up, dXp, dw, dGz, cx, cvq, part, total;
+};
+
+static BwdCarve carve_backward(const Dims& d) {
+  BwdCarve c{};
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    const size_t at = off;
+    off += align_up(bytes > 0 ? bytes : 1);
+    return at;
+  };
+  const size_t es = elem_size(d.dtype);
+  const size_t R = (size_t)d.N + 2 * (size_t)d.n_const;
+  c.dYp = take(es * (size_t)d.M_cap * d.D);
+  c.gate = take(es * (size_t)d.M_cap * d.F);
+  c.up = take(es * (size_t)d.M_cap * d.F);
+  c.dXp = take(es * (size_t)d.M_cap * d.D);
+  c.dw = take(sizeof(float) * (size_t)d.T * d.K);
+  c.dGz = take(sizeof(float) * (size_t)d.T * R);
+  c.cx = take(sizeof(float) * (size_t)d.T);
+  c.cvq = take(sizeof(float) * (size_t)d.T * d.n_const);
+  const size_t widest = R * (size_t)d.D > (size_t)d.N * d.N ? R * (size_t)d.D : (size_t)d.N * d.N;
+  c.part = take(sizeof(float) * widest * (size_t)backward_token_chunks(d, nullptr));
+  c.total = off;
+  return c;
+}
+
+moepp_status moepp_backward_workspace_bytes(const moepp_config* cfg, size_t* bytes) {
+  Dims d;
+  const moepp_status s = make_dims(cfg, &d);
+  if (s != MOEPP_OK) return s;
+  if (bytes == nullptr) return MOEPP_ERR_INVALID_ARG;
+  *bytes = carve_backward(d).total;
+  return MOEPP_OK;
+}
+
+moepp_status moepp_layer_backward(const moepp_config* cfg, const moepp_weights* weights, const void* x,
+                                  const float* prev_logits, const float* logits, const void* dy,
+                                  const float* dlogits_next, const void* fwd_workspace, size_t fwd_workspace_bytes,
+                                  const moepp_grads* grads, void* bwd_workspace, size_t bwd_workspace_bytes,
+                                  void* stream) {
+  Dims d;
+  moepp_status s = make_dims(cfg, &d);
+  if (s != MOEPP_OK) return s;
+  if (grads == nullptr || bwd_workspace == nullptr) return MOEPP_ERR_INVALID_ARG;
+  if (d.flags & MOEPP_FLAG_FUSED_GATHER) return MOEPP_ERR_INVALID_ARG;
+  s = check_layer_args(d, weights, x, prev_logits, dy, fwd_workspace);
+  if (s != MOEPP_OK) return s;
+  const moepp_grads& g = *grads;
+  if (g.dW_r == nullptr || (d.T > 0 && g.dx == nullptr)) return MOEPP_ERR_INVALID_ARG;
+  if (d.T > 0 && weights->W_g != nullptr && g.dprev == nullptr) return MOEPP_ERR_INVALID_ARG;
+  if (d.n_const > 0 && (g.dW_c == nullptr || g.dv == nullptr)) return MOEPP_ERR_INVALID_ARG;
+  if (d.n_ffn > 0 && (g.dW_gate == nullptr || g.dW_up == nullptr || g.dW_down == nullptr))
+    return MOEPP_ERR_INVALID_ARG;
+  if (!aligned16(dy) || !aligned16(g.dx) || !aligned16(x)) return MOEPP_ERR_ALIGN;
+  if ((reinterpret_cast<uintptr_t>(bwd_workspace) & (kAlign - 1)) != 0) return MOEPP_ERR_ALIGN;
+  const Carve c = carve(d, false);
+  const BwdCarve bc = carve_backward(d);
+  if (fwd_workspace_bytes < c.total || bwd_workspace_bytes < bc.total) return MOEPP_ERR_WORKSPACE;
+  const char* fw = static_cast<const char*>(fwd_workspace);
+  char* bw = static_cast<char*>(bwd_workspace);
+  ForwardState fs{};
+  fs.logits = logits != nullptr ? logits : reinterpret_cast<const float*>(fw + c.logits);
+  fs.topk_idx = reinterpret_cast<const int32_t*>(fw + c.topk_idx);
+  fs.topk_w = reinterpret_cast<const float*>(fw + c.topk_w);
+  fs.offsets = reinterpret_cast<const int32_t*>(fw + c.offsets);
+  fs.alpha = reinterpret_cast<const float*>(fw + c.alpha);
+  fs.row_of_slot = reinterpret_cast<const int32_t*>(fw + c.row_of_slot);
+  fs.slot_of_row = reinterpret_cast<const int32_t*>(fw + c.slot_of_row);
+  fs.x_perm = fw + c.x_perm;
+  fs.h = fw + c.h;
+  fs.y_perm = fw + c.y_perm;
+  BackwardScratch b{};
+  b.dYp = bw + bc.dYp; b.gate = bw + bc.gate; b.up = bw + bc.up; b.dXp = bw + bc.dXp;
+  b.dw = reinterpret_cast<float*>(bw + bc.dw);
+  b.dGz = reinterpret_cast<float*>(bw + bc.dGz);
+  b.cx = reinterpret_cast<float*>(bw + bc.cx);
+  b.cvq = reinterpret_cast<float*>(bw + bc.cvq);
+  b.part = reinterpret_cast<float*>(bw + bc.part);
+  return from_cuda(launch_layer_backward(d, fs, *weights, x, prev_logits, dy, dlogits_next, b, g,
+                                         static_cast<cudaStream_t>(stream)));
+}
+
 moepp_status moepp_device_error(int32_t* code) {
   if (code == nullptr) return MOEPP_ERR_INVALID_ARG;
   const cudaError_t e = read_and_clear_device_error(code);

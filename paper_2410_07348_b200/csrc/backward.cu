@@ -1,0 +1,419 @@
+// Backward pass of the layer outside the expert GEMMs: the chain rule through the combine (Eq. 1, Eq. 3-5), the
+// gate (Eq. 1) and the router with its gating residual (Eq. 2, Eq. 6), with the picks held fixed.
+//   combine_bwd : per token, dL/dE_k = w_k dy scattered to the grouped rows, dL/dw_k = <dy, E_k(x)>, the
+//                 coefficient of dy that flows straight to x, and the constant experts' mixing gradients
+//   gate_bwd    : dL/dG through the softmax over all N experts (and the optional renormalisation), plus the
+//                 gradient the next layer sends back through its gating residual; dL/dG_prev = dG W_g
+//   token_outer : sum over tokens of a[t, :]^T b[t, :] in fixed chunks (deterministic two-stage reduction),
+//                 used for dW_r, dW_c, dW_g, dv
+//   dx_assemble : dx = cx dy + [dG | dz] [W_r ; W_c] + the K grouped rows of dXp
+#include "common.cuh"
+
+namespace moepp {
+namespace {
+
+constexpr int kWarpsPerBlock = 8;
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// One warp per token.
+//   dYp[row_k, :] = w_k dy            (FFN picks that were kept)
+//   dw[t, k]      = <dy, E_k(x)>      (0 for zero experts and dropped slots)
+//   cx[t]         = residual + sum of w_k over copy picks + sum of w_k a1 over constant picks
+//   cvq[t, q]     = w_k a2 for the constant expert q the token picked, else 0
+//   dGz[t, N + 2q + j] = dL/dz_j of constant expert q's mixing logits, else 0
+template <typename XT>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+combine_bwd_kernel(Dims dm, int R, const XT* __restrict__ x, const XT* __restrict__ dy,
+                   const XT* __restrict__ y_perm, const int32_t* __restrict__ topk_idx,
+                   const float* __restrict__ topk_w, const int32_t* __restrict__ row_of_slot,
+                   const float* __restrict__ alpha, const float* __restrict__ v, XT* __restrict__ dYp,
+                   float* __restrict__ dw, float* __restrict__ cx_out, float* __restrict__ cvq,
+                   float* __restrict__ dGz) {
+  const int lane = threadIdx.x & 31;
+  const long long t = (long long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+  if (t >= dm.T) return;
+  const int K = dm.K, D = dm.D, N = dm.N;
+  const int zero0 = dm.zero0(), copy0 = dm.copy0(), const0 = dm.const0();
+  const XT* xt = x + (size_t)t * D;
+  const XT* dyt = dy + (size_t)t * D;
+
+  for (int i = lane; i < 2 * dm.n_const; i += 32) dGz[t * R + N + i] = 0.f;
+  for (int i = lane; i < dm.n_const; i += 32) cvq[t * dm.n_const + i] = 0.f;
+  __syncwarp();
+
+  float cx = dm.add_residual ? 1.f : 0.f;
+  float dyx = 0.f;
+  bool have_dyx = false;
+  for (int k = 0; k < K; ++k) {
+    const int e = topk_idx[t * K + k];
+    const float g = topk_w[t * K + k];
+    const int row = row_of_slot[t * K + k];
+    float dwk = 0.f;
+    if (row == -2 || (e >= zero0 && e < copy0)) {
+      // dropped (Eq. 8) or a zero expert (Eq. 3): nothing flows
+    } else if (e < zero0) {
+      float acc = 0.f;
+      for (int d = lane * 8; d < D; d += 256) {
+        float dv8[8], yv[8], o[8];
+        Vec8<XT>::load(dyt + d, dv8);
+        Vec8<XT>::load(y_perm + (size_t)row * D + d, yv);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          acc = fmaf(dv8[i], yv[i], acc);
+          o[i] = g * dv8[i];
+        }
+        Vec8<XT>::store(dYp + (size_t)row * D + d, o);
+      }
+      dwk = warp_sum(acc);
+    } else {
+      if (!have_dyx) {
+        float acc = 0.f;
+        for (int d = lane * 8; d < D; d += 256) {
+          float dv8[8], xv[8];
+          Vec8<XT>::load(dyt + d, dv8);
+          Vec8<XT>::load(xt + d, xv);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) acc = fmaf(dv8[i], xv[i], acc);
+        }
+        dyx = warp_sum(acc);
+        have_dyx = true;
+      }
+      if (e < const0) {  // Eq. 4
+        dwk = dyx;
+        cx += g;
+      } else {  // Eq. 5
+        const int q = e - const0;
+        const float a1 = alpha[(t * dm.n_const + q) * 2 + 0], a2 = alpha[(t * dm.n_const + q) * 2 + 1];
+        float acc = 0.f;
+        for (int d = lane * 8; d < D; d += 256) {
+          float dv8[8];
+          Vec8<XT>::load(dyt + d, dv8);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) acc = fmaf(dv8[i], __ldg(v + (size_t)q * D + d + i), acc);
+        }
+        const float dyv = warp_sum(acc);
+        dwk = a1 * dyx + a2 * dyv;
+        const float da1 = g * dyx, da2 = g * dyv, mean = a1 * da1 + a2 * da2;
+        cx += g * a1;
+        if (lane == 0) {
+          cvq[t * dm.n_const + q] = g * a2;
+          dGz[t * R + N + 2 * q + 0] = a1 * (da1 - mean);
+          dGz[t * R + N + 2 * q + 1] = a2 * (da2 - mean);
+        }
+      }
+    }
+    if (lane == 0) dw[t * K + k] = dwk;
+  }
+  if (lane == 0) cx_out[t] = cx;
+}
+
+// Grouped rows no slot owns (padding up to row_align) get a zero gradient, so they add nothing to the GEMMs.
+template <typename XT>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+zero_pad_rows_kernel(const int32_t* __restrict__ slot_of_row, const int32_t* __restrict__ offsets, int n_ffn, int D,
+                     XT* __restrict__ dYp) {
+  const int lane = threadIdx.x & 31;
+  const long long row = (long long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+  if (row >= offsets[n_ffn] || slot_of_row[row] >= 0) return;
+  const float z[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  for (int d = lane * 8; d < D; d += 256) Vec8<XT>::store(dYp + (size_t)row * D + d, z);
+}
+
+// One warp per token; lane l holds experts l and l + 32.
+//   P = softmax(logits[t, :]);  w_k = P[idx_k] (/ S, the sum over the picks, if renormalised)
+//   dP[idx_k] = dw_k                      or (dw_k - sum_j dw_j w_j) / S when renormalised
+//   dG = P (dP - <dP, P>) + dlogits_next;  dprev = dG W_g
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+gate_bwd_kernel(Dims dm, int R, const float* __restrict__ logits, const int32_t* __restrict__ topk_idx,
+                const float* __restrict__ topk_w, const float* __restrict__ dw,
+                const float* __restrict__ dlogits_next, const float* __restrict__ W_g, float* __restrict__ dGz,
+                float* __restrict__ dprev) {
+  extern __shared__ float s_Wg[];  // [N, N] when W_g is given
+  const int N = dm.N, K = dm.K;
+  if (W_g != nullptr) {
+    for (int i = threadIdx.x; i < N * N; i += blockDim.x) s_Wg[i] = W_g[i];
+    __syncthreads();
+  }
+  const int lane = threadIdx.x & 31;
+  const long long t = (long long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+  if (t >= dm.T) return;
+  const int i0 = lane, i1 = lane + 32;
+  const float g0 = i0 < N ? logits[t * N + i0] : -INFINITY;
+  const float g1 = i1 < N ? logits[t * N + i1] : -INFINITY;
+  float m = fmaxf(g0, g1);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  const float e0 = i0 < N ? expf(g0 - m) : 0.f, e1 = i1 < N ? expf(g1 - m) : 0.f;
+  const float inv = 1.f / warp_sum(e0 + e1);
+  const float P0 = e0 * inv, P1 = e1 * inv;
+
+  // lane k holds pick k
+  int e_l = -1;
+  float dw_l = 0.f, w_l = 0.f;
+  if (lane < K) {
+    e_l = topk_idx[t * K + lane];
+    dw_l = dw[t * K + lane];
+    w_l = topk_w[t * K + lane];
+  }
+  float dot = 0.f, S = 1.f;
+  if (dm.renorm) {
+    dot = warp_sum(dw_l * w_l);
+    float sp = 0.f;
+    for (int k = 0; k < K; ++k) {
+      const int e = __shfl_sync(0xffffffffu, e_l, k);
+      sp += (e == i0 ? P0 : 0.f) + (e == i1 ? P1 : 0.f);
+    }
+    S = warp_sum(sp);
+  }
+  float dP0 = 0.f, dP1 = 0.f;
+  for (int k = 0; k < K; ++k) {
+    const int e = __shfl_sync(0xffffffffu, e_l, k);
+    const float dk = __shfl_sync(0xffffffffu, dw_l, k);
+    const float val = dm.renorm ? (dk - dot) / S : dk;
+    if (e == i0) dP0 += val;
+    if (e == i1) dP1 += val;
+  }
+  const float dotP = warp_sum(dP0 * P0 + dP1 * P1);
+  float dG0 = P0 * (dP0 - dotP), dG1 = P1 * (dP1 - dotP);
+  if (dlogits_next != nullptr) {
+    if (i0 < N) dG0 += dlogits_next[t * N + i0];
+    if (i1 < N) dG1 += dlogits_next[t * N + i1];
+  }
+  if (i0 < N) dGz[t * R + i0] = dG0;
+  if (i1 < N) dGz[t * R + i1] = dG1;
+  if (W_g != nullptr) {  // Eq. 6: G = ... + W_g G_prev
+    float a0 = 0.f, a1 = 0.f;
+    for (int i = 0; i < N; ++i) {
+      const float gi = __shfl_sync(0xffffffffu, i < 32 ? dG0 : dG1, i & 31);
+      if (i0 < N) a0 = fmaf(gi, s_Wg[i * N + i0], a0);
+      if (i1 < N) a1 = fmaf(gi, s_Wg[i * N + i1], a1);
+    }
+    if (i0 < N) dprev[t * N + i0] = a0;
+    if (i1 < N) dprev[t * N + i1] = a1;
+  }
+}
+
+constexpr int kOm = 64, kOn = 64, kOk = 16;
+
+__device__ __forceinline__ float ldf(const float* p) { return *p; }
+__device__ __forceinline__ float ldf(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+
+// part[z, m, n] = sum over the tokens t of chunk z of A[t, m] * B[t, n]   (A float [T, M], B [T, Nout])
+template <typename TB>
+__global__ void __launch_bounds__(256)
+token_outer_kernel(const float* __restrict__ A, const TB* __restrict__ B, float* __restrict__ part, int T, int M,
+                   int Nout, long long a_rs, long long b_rs, int chunk) {
+  __shared__ float As[kOk][kOm + 4], Bs[kOk][kOn + 4];
+  const int m0 = blockIdx.x * kOm, n0 = blockIdx.y * kOn, z = blockIdx.z;
+  const int t_begin = z * chunk, t_end = min(T, t_begin + chunk);
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  float acc[4][4] = {};
+  for (int t0 = t_begin; t0 < t_end; t0 += kOk) {
+    __syncthreads();
+    for (int i = tid; i < kOm * kOk; i += 256) {
+      const int m = i % kOm, k = i / kOm;
+      As[k][m] = (t0 + k < t_end && m0 + m < M) ? A[(size_t)(t0 + k) * a_rs + m0 + m] : 0.f;
+    }
+    for (int i = tid; i < kOn * kOk; i += 256) {
+      const int n = i % kOn, k = i / kOn;
+      Bs[k][n] = (t0 + k < t_end && n0 + n < Nout) ? ldf(B + (size_t)(t0 + k) * b_rs + n0 + n) : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < kOk; ++kk) {
+      const float4 av = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);
+      const float4 bv = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
+      const float am[4] = {av.x, av.y, av.z, av.w}, bm[4] = {bv.x, bv.y, bv.z, bv.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(am[i], bm[j], acc[i][j]);
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int m = m0 + ty * 4 + i, n = n0 + tx * 4 + j;
+      if (m < M && n < Nout) part[((size_t)z * M + m) * Nout + n] = acc[i][j];
+    }
+}
+
+// out[i] = sum over z (in order) of part[z, i]
+__global__ void __launch_bounds__(256) sum_parts_kernel(const float* __restrict__ part, float* __restrict__ out,
+                                                        long long n, int Z) {
+  const long long i = (long long)blockIdx.x * 256 + threadIdx.x;
+  if (i >= n) return;
+  float s = 0.f;
+  for (int z = 0; z < Z; ++z) s += part[(size_t)z * n + i];
+  out[i] = s;
+}
+
+// out[i] = sum over tokens of A[t, i]; one block per column, fixed order of the partial sums
+__global__ void __launch_bounds__(256) column_sum_kernel(const float* __restrict__ A, float* __restrict__ out, int T,
+                                                         long long a_rs) {
+  __shared__ float s[256];
+  float acc = 0.f;
+  for (int t = threadIdx.x; t < T; t += 256) acc += A[(size_t)t * a_rs + blockIdx.x];
+  s[threadIdx.x] = acc;
+  __syncthreads();
+  for (int o = 128; o > 0; o >>= 1) {
+    if ((int)threadIdx.x < o) s[threadIdx.x] += s[threadIdx.x + o];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) out[blockIdx.x] = s[0];
+}
+
+// One warp per token: dx = cx dy + sum_r dGz[t, r] Wrow_r + sum over kept FFN picks of dXp[row_k, :],
+// Wrow_r = W_r[r, :] for r < N and the flattened W_c rows after that.
+template <typename XT>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+dx_assemble_kernel(Dims dm, int R, const XT* __restrict__ dy, const float* __restrict__ cx,
+                   const float* __restrict__ dGz, const float* __restrict__ W_r, const float* __restrict__ W_c,
+                   const XT* __restrict__ dXp, const int32_t* __restrict__ topk_idx,
+                   const int32_t* __restrict__ row_of_slot, XT* __restrict__ dx) {
+  __shared__ float s_c[kWarpsPerBlock][kMaxRouteRows];
+  const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+  const long long t = (long long)blockIdx.x * kWarpsPerBlock + wib;
+  if (t >= dm.T) return;
+  const int D = dm.D, N = dm.N, K = dm.K;
+  for (int r = lane; r < R; r += 32) s_c[wib][r] = dGz[t * R + r];
+  int rows[kMaxTopK];
+#pragma unroll
+  for (int k = 0; k < kMaxTopK; ++k) {
+    rows[k] = -1;
+    if (k < K && topk_idx[t * K + k] < dm.n_ffn) rows[k] = row_of_slot[t * K + k];  // -2 when dropped
+  }
+  __syncwarp();
+  const float c = cx[t];
+  for (int d = lane * 8; d < D; d += 256) {
+    float acc[8], tmp[8];
+    Vec8<XT>::load(dy + (size_t)t * D + d, tmp);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[i] = c * tmp[i];
+    for (int r = 0; r < R; ++r) {
+      const float g = s_c[wib][r];
+      const float* wrow = r < N ? W_r + (size_t)r * D + d : W_c + (size_t)(r - N) * D + d;
+      const float4 a = __ldg(reinterpret_cast<const float4*>(wrow));
+      const float4 b = __ldg(reinterpret_cast<const float4*>(wrow + 4));
+      acc[0] = fmaf(g, a.x, acc[0]); acc[1] = fmaf(g, a.y, acc[1]); acc[2] = fmaf(g, a.z, acc[2]);
+      acc[3] = fmaf(g, a.w, acc[3]); acc[4] = fmaf(g, b.x, acc[4]); acc[5] = fmaf(g, b.y, acc[5]);
+      acc[6] = fmaf(g, b.z, acc[6]); acc[7] = fmaf(g, b.w, acc[7]);
+    }
+#pragma unroll
+    for (int k = 0; k < kMaxTopK; ++k) {
+      if (rows[k] >= 0) {
+        Vec8<XT>::load(dXp + (size_t)rows[k] * D + d, tmp);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[i] += tmp[i];
+      }
+    }
+    Vec8<XT>::store(dx + (size_t)t * D + d, acc);
+  }
+}
+
+}  // namespace
+
+// The reductions over tokens run in at most 64 chunks of at least 512 tokens.
+int backward_token_chunks(const Dims& d, int* chunk_tokens) {
+  int chunk = (d.T + 63) / 64;
+  if (chunk < 512) chunk = 512;
+  chunk = (chunk + kOk - 1) / kOk * kOk;
+  if (chunk_tokens != nullptr) *chunk_tokens = chunk;
+  return d.T > 0 ? (d.T + chunk - 1) / chunk : 1;
+}
+
+namespace {
+
+template <typename TB>
+cudaError_t token_outer(const Dims& d, const float* A, long long a_rs, int M, const TB* B, long long b_rs, int Nout,
+                        float* part, float* out, cudaStream_t st) {
+  if (M == 0 || Nout == 0) return cudaSuccess;
+  int chunk;
+  const int Z = backward_token_chunks(d, &chunk);
+  dim3 grid((unsigned)((M + kOm - 1) / kOm), (unsigned)((Nout + kOn - 1) / kOn), (unsigned)Z);
+  token_outer_kernel<TB><<<grid, 256, 0, st>>>(A, B, part, d.T, M, Nout, a_rs, b_rs, chunk);
+  cudaError_t err = cudaGetLastError();
+  if (err != cudaSuccess) return err;
+  const long long n = (long long)M * Nout;
+  sum_parts_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(part, out, n, Z);
+  return cudaGetLastError();
+}
+
+template <typename XT>
+cudaError_t layer_backward_t(const Dims& d, const ForwardState& fs, const moepp_weights& w, const XT* x,
+                             const float* prev, const XT* dy, const float* dlogits_next, const BackwardScratch& b,
+                             const moepp_grads& g, cudaStream_t st) {
+  const int R = d.N + 2 * d.n_const;
+  const unsigned token_blocks = (unsigned)((d.T + kWarpsPerBlock - 1) / kWarpsPerBlock);
+  cudaError_t err;
+  combine_bwd_kernel<XT><<<token_blocks, kWarpsPerBlock * 32, 0, st>>>(
+      d, R, x, dy, static_cast<const XT*>(fs.y_perm), fs.topk_idx, fs.topk_w, fs.row_of_slot, fs.alpha, w.v,
+      static_cast<XT*>(b.dYp), b.dw, b.cx, b.cvq, b.dGz);
+  if ((err = cudaGetLastError()) != cudaSuccess) return err;
+  if (d.n_ffn > 0 && d.M_cap > 0 && d.row_align > 1) {
+    zero_pad_rows_kernel<XT><<<(unsigned)((d.M_cap + kWarpsPerBlock - 1) / kWarpsPerBlock), kWarpsPerBlock * 32, 0,
+                               st>>>(fs.slot_of_row, fs.offsets, d.n_ffn, d.D, static_cast<XT*>(b.dYp));
+    if ((err = cudaGetLastError()) != cudaSuccess) return err;
+  }
+  const size_t wg_smem = w.W_g != nullptr ? sizeof(float) * (size_t)d.N * d.N : 0;
+  gate_bwd_kernel<<<token_blocks, kWarpsPerBlock * 32, wg_smem, st>>>(d, R, fs.logits, fs.topk_idx, fs.topk_w, b.dw,
+                                                                       dlogits_next, w.W_g, b.dGz, g.dprev);
+  if ((err = cudaGetLastError()) != cudaSuccess) return err;
+
+  err = launch_ffn_backward_simt(d, fs.x_perm, fs.offsets, w.W_gate, w.W_up, w.W_down, fs.h, b.dYp, b.gate, b.up,
+                                 b.dXp, g.dW_gate, g.dW_up, g.dW_down, st);
+  if (err != cudaSuccess) return err;
+
+  // router and constant-expert weights: [dG | dz]^T x, rows 0..N-1 -> dW_r, the rest -> dW_c
+  // (both land in one [R, D] product; it is computed into `part` and split on the way out)
+  if ((err = token_outer<XT>(d, b.dGz, R, d.N, x, d.D, d.D, b.part, g.dW_r, st)) != cudaSuccess) return err;
+  if (d.n_const > 0) {
+    if ((err = token_outer<XT>(d, b.dGz + d.N, R, 2 * d.n_const, x, d.D, d.D, b.part, g.dW_c, st)) != cudaSuccess)
+      return err;
+    if ((err = token_outer<XT>(d, b.cvq, d.n_const, d.n_const, dy, d.D, d.D, b.part, g.dv, st)) != cudaSuccess)
+      return err;
+  }
+  if (w.W_g != nullptr && g.dW_g != nullptr) {
+    if ((err = token_outer<float>(d, b.dGz, R, d.N, prev, d.N, d.N, b.part, g.dW_g, st)) != cudaSuccess) return err;
+  }
+  if (g.dbias != nullptr) {
+    column_sum_kernel<<<(unsigned)d.N, 256, 0, st>>>(b.dGz, g.dbias, d.T, R);
+    if ((err = cudaGetLastError()) != cudaSuccess) return err;
+  }
+  dx_assemble_kernel<XT><<<token_blocks, kWarpsPerBlock * 32, 0, st>>>(
+      d, R, dy, b.cx, b.dGz, w.W_r, w.W_c, static_cast<const XT*>(b.dXp), fs.topk_idx, fs.row_of_slot,
+      static_cast<XT*>(g.dx));
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_layer_backward(const Dims& d, const ForwardState& fs, const moepp_weights& w, const void* x,
+                                  const float* prev, const void* dy, const float* dlogits_next,
+                                  const BackwardScratch& b, const moepp_grads& g, cudaStream_t st) {
+  if (d.T == 0) {  // no tokens: every weight gradient is zero
+    const int R2 = 2 * d.n_const;
+    cudaError_t err;
+    auto zero = [&](float* p, size_t n) { return (p == nullptr || n == 0) ? cudaSuccess : cudaMemsetAsync(p, 0, sizeof(float) * n, st); };
+    if ((err = zero(g.dW_r, (size_t)d.N * d.D)) != cudaSuccess) return err;
+    if ((err = zero(g.dW_g, (size_t)d.N * d.N)) != cudaSuccess) return err;
+    if ((err = zero(g.dbias, (size_t)d.N)) != cudaSuccess) return err;
+    if ((err = zero(g.dW_c, (size_t)R2 * d.D)) != cudaSuccess) return err;
+    if ((err = zero(g.dv, (size_t)d.n_const * d.D)) != cudaSuccess) return err;
+    return launch_ffn_backward_simt(d, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr,
+                                    nullptr, g.dW_gate, g.dW_up, g.dW_down, st);
+  }
+  return d.dtype == MOEPP_BF16
+             ? layer_backward_t<__nv_bfloat16>(d, fs, w, static_cast<const __nv_bfloat16*>(x), prev,
+                                               static_cast<const __nv_bfloat16*>(dy), dlogits_next, b, g, st)
+             : layer_backward_t<float>(d, fs, w, static_cast<const float*>(x), prev, static_cast<const float*>(dy),
+                                       dlogits_next, b, g, st);
+}
+
+}  // namespace moepp

@@ -64,6 +64,43 @@ cudaError_t launch_combine(const Dims& d, const void* x, const void* y_perm, con
                            const float* topk_w, const int32_t* row_of_slot, const float* alpha, const float* W_c,
                            const float* v, void* y, cudaStream_t st);
 
+// ---- backward pass ---------------------------------------------------------------------------------
+// What the forward pass left in its workspace (all device pointers).
+struct ForwardState {
+  const float* logits;
+  const int32_t* topk_idx;
+  const float* topk_w;
+  const int32_t* offsets;
+  const float* alpha;
+  const int32_t* row_of_slot;
+  const int32_t* slot_of_row;
+  const void* x_perm;
+  const void* h;
+  const void* y_perm;
+};
+
+// Device scratch of one backward pass.
+struct BackwardScratch {
+  void *dYp, *gate, *up, *dXp;  // grouped rows, activation dtype: [M_cap, D], [M_cap, F] x 2, [M_cap, D]
+  float* dw;                    // [T, K]
+  float* dGz;                   // [T, R], R = N + 2 n_const: dL/dlogits, then dL/d(mixing logits)
+  float* cx;                    // [T]
+  float* cvq;                   // [T, n_const]
+  float* part;                  // [chunks, max(R D, N N)] partial sums of the reductions over tokens
+};
+
+int backward_token_chunks(const Dims& d, int* chunk_tokens);
+
+cudaError_t launch_ffn_backward_simt(const Dims& d, const void* x_perm, const int32_t* offsets, const void* W_gate,
+                                     const void* W_up, const void* W_down, const void* h, const void* dy_perm,
+                                     void* gate_buf, void* up_buf, void* dx_perm, float* dW_gate, float* dW_up,
+                                     float* dW_down, cudaStream_t st);
+
+// Whole backward pass of one layer; grads are overwritten.
+cudaError_t launch_layer_backward(const Dims& d, const ForwardState& fs, const moepp_weights& w, const void* x,
+                                  const float* prev, const void* dy, const float* dlogits_next,
+                                  const BackwardScratch& b, const moepp_grads& g, cudaStream_t st);
+
 // Error word written by kernels whose bounded waits ran out (0 = fine).
 cudaError_t read_and_clear_device_error(int32_t* code);
 int32_t* device_error_word();  // device address of that word on the current device (nullptr on failure)

@@ -1,0 +1,120 @@
+"""GPU parity of the layer's backward pass (moepp_layer_backward) against the CPU oracle, through the C-ABI.
+
+The forward call fills its workspace, the backward call reads it; the oracle differentiates the same layer in
+float64 with the GPU's own picks held fixed.  Every gradient tensor is compared element by element, the error
+measured against that tensor's largest magnitude: float32 storage within 2e-4, bf16 storage within 2e-2 (the
+grouped intermediates dL/dE, the SwiGLU pre-activations and their gradients are rounded to bf16 on the way).
+"""
+import numpy as np
+import pytest
+import torch
+
+from harness import f32, oracle_inputs, shape_of
+from paper_2410_07348_b200 import binding as B
+from paper_2410_07348_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"f32": 2e-4, "bf16": 2e-2}
+GRADS = ("dx", "dprev", "dW_r", "dW_g", "dbias", "dW_c", "dv", "dW_gate", "dW_up", "dW_down")
+
+
+def gpu_backward(cfg, wd, x, prev, dy, dlogits):
+    T, N, K = cfg.T, cfg.N, cfg.top_k
+    dev = "cuda"
+    ws = torch.empty(B.moepp_workspace_bytes(cfg), dtype=torch.uint8, device=dev)
+    y = torch.empty(T, cfg.D, dtype=x.dtype, device=dev)
+    logits = torch.empty(T, N, device=dev)
+    B.moepp_layer_forward(cfg, wd, x, prev, y, logits, ws)
+    idx = torch.empty(T, K, dtype=torch.int32, device=dev)
+    w = torch.empty(T, K, device=dev)
+    counts = torch.empty(N, dtype=torch.int32, device=dev)
+    offsets = torch.empty(cfg.n_ffn + 1, dtype=torch.int32, device=dev)
+    lg2 = torch.empty(T, N, device=dev)
+    B.moepp_route(cfg, x, wd["W_r"], wd["W_g"], prev, wd["router_bias"], None, lg2, idx, w, counts, offsets, None)
+    nan = lambda *shape, dtype=torch.float32: torch.full(shape, float("nan"), dtype=dtype, device=dev)
+    g = dict(dx=nan(T, cfg.D, dtype=x.dtype), dprev=nan(T, N) if prev is not None else None, dW_r=nan(N, cfg.D),
+             dW_g=nan(N, N) if prev is not None else None, dbias=nan(N), dW_c=nan(max(cfg.n_const, 1), 2, cfg.D),
+             dv=nan(max(cfg.n_const, 1), cfg.D), dW_gate=nan(max(cfg.n_ffn, 1), cfg.F, cfg.D),
+             dW_up=nan(max(cfg.n_ffn, 1), cfg.F, cfg.D), dW_down=nan(max(cfg.n_ffn, 1), cfg.D, cfg.F))
+    bws = torch.empty(B.moepp_backward_workspace_bytes(cfg), dtype=torch.uint8, device=dev)
+    B.moepp_layer_backward(cfg, wd, x, prev, logits, dy, dlogits, ws, g, bws)
+    torch.cuda.synchronize()
+    assert B.moepp_device_error() == 0
+    return {k: (None if v is None else v.float().cpu().numpy()) for k, v in g.items()}, idx.cpu().numpy()
+
+
+def check_backward(oracle64, lt, seed=0, with_dlogits=True, **over):
+    spec = lt.spec
+    cfg = B.config_from_spec(spec, **over)
+    wd = B.weights_from_tensors(lt)
+    x, prev = lt.x.cuda(), None if lt.prev is None else lt.prev.cuda()
+    gen = torch.Generator().manual_seed(77 + seed)
+    dy = torch.randn(spec.T, spec.D, generator=gen).to(x.dtype)
+    dlogits = (0.1 * torch.randn(spec.T, spec.N, generator=gen)) if with_dlogits else None
+    got, idx_g = gpu_backward(cfg, wd, x, prev, dy.cuda(), None if dlogits is None else dlogits.cuda())
+    s = shape_of(spec, **{k: v for k, v in over.items()
+                          if k in ("renorm_topk", "row_align", "add_residual", "tau", "capacity_factor")})
+    oi = oracle_inputs(lt)
+    ref = oracle64.layer_backward(s, oi["x"], oi["W_r"], idx_g, f32(dy), oi["W_g"], oi["prev"], oi["bias"], oi["W_c"],
+                                  oi["v"], f32(lt.W_gate), f32(lt.W_up), f32(lt.W_down), dlogits=f32(dlogits))
+    tol = TOL[spec.dtype]
+    worst = {}
+    for name in GRADS:
+        r = ref[name]
+        if r is None or r.size == 0 or got[name] is None:
+            continue
+        gq = got[name].reshape(-1)[:r.size].reshape(r.shape)
+        assert np.isfinite(gq).all(), name
+        scale = max(float(np.abs(r).max()), 1e-6)
+        worst[name] = float(np.abs(gq.astype(np.float64) - r).max()) / scale
+        assert worst[name] <= tol, (name, worst[name], scale)
+    return worst
+
+
+def test_backward_cfg1_f32(oracle64):
+    lt = W.make_config("cfg1_tiny_f32")
+    check_backward(oracle64, lt)
+    check_backward(oracle64, lt, renorm_topk=1, add_residual=1, row_align=128)
+    check_backward(oracle64, lt, with_dlogits=False)
+
+
+def test_backward_first_layer_vanilla(oracle64):
+    lt = W.make_layer(W.CONFIGS["cfg1_tiny_f32"].vanilla(), seed=0, with_prev=False)
+    check_backward(oracle64, lt)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_backward_several_tiles(oracle64, dtype):
+    """Several 64-row tiles per expert with ragged tails, all four expert kinds, padded segments."""
+    spec = W.LayerSpec(T=1900, D=264, F=392, n_ffn=5, n_zero=1, n_copy=1, n_const=2, top_k=2, dtype=dtype)
+    lt = W.make_layer(spec, seed=3, with_prev=True, w_std=0.05)
+    check_backward(oracle64, lt, row_align=128, add_residual=1)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_backward_random_shapes(oracle64, seed):
+    rng = np.random.default_rng(2000 + seed)
+    dtype = "bf16" if seed % 2 == 0 else "f32"
+    n_ffn = int(rng.integers(1, 9))
+    n_zero, n_copy, n_const = int(rng.integers(0, 3)), int(rng.integers(0, 3)), int(rng.integers(0, 4))
+    N = n_ffn + n_zero + n_copy + n_const
+    spec = W.LayerSpec(T=int(rng.integers(1, 900)), D=8 * int(rng.integers(1, 40)), F=8 * int(rng.integers(1, 40)),
+                       n_ffn=n_ffn, n_zero=n_zero, n_copy=n_copy, n_const=n_const,
+                       top_k=int(rng.integers(1, min(N, 4) + 1)), dtype=dtype)
+    lt = W.make_layer(spec, seed=seed, with_prev=bool(seed & 2), w_std=0.05)
+    over = dict(row_align=int(rng.choice([1, 8, 128])), add_residual=int(rng.integers(0, 2)),
+                renorm_topk=int(rng.integers(0, 2)))
+    if seed % 3 == 0:
+        over.update(capacity_factor=float(rng.choice([0.7, 1.1])), tau=float(rng.choice([0.5, 0.75, 1.0])))
+    check_backward(oracle64, lt, seed=seed, **over)
+
+
+def test_backward_no_tokens():
+    spec = W.LayerSpec(T=0, D=64, F=96, n_ffn=2, n_zero=1, n_copy=1, n_const=1, top_k=2, dtype="f32")
+    lt = W.make_layer(spec, seed=0, with_prev=True)
+    cfg = B.config_from_spec(spec)
+    wd = B.weights_from_tensors(lt)
+    got, _ = gpu_backward(cfg, wd, lt.x.cuda(), lt.prev.cuda(), torch.empty(0, 64, device="cuda"), None)
+    for name in GRADS[2:]:
+        assert not np.any(got[name]), name
