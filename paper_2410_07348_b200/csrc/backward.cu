@@ -366,8 +366,13 @@ cudaError_t layer_backward_t(const Dims& d, const ForwardState& fs, const moepp_
                                                                        dlogits_next, w.W_g, b.dGz, g.dprev);
   if ((err = cudaGetLastError()) != cudaSuccess) return err;
 
-  err = launch_ffn_backward_simt(d, fs.x_perm, fs.offsets, w.W_gate, w.W_up, w.W_down, fs.h, b.dYp, b.gate, b.up,
+  err = cudaErrorNotSupported;
+  if (!(d.flags & MOEPP_FLAG_SIMT_FFN))
+    err = launch_ffn_backward_tc(d, fs.x_perm, fs.offsets, w.W_gate, w.W_up, w.W_down, fs.h, b.dYp, b.gate, b.up,
                                  b.dXp, g.dW_gate, g.dW_up, g.dW_down, st);
+  if (err == cudaErrorNotSupported)
+    err = launch_ffn_backward_simt(d, fs.x_perm, fs.offsets, w.W_gate, w.W_up, w.W_down, fs.h, b.dYp, b.gate, b.up,
+                                   b.dXp, g.dW_gate, g.dW_up, g.dW_down, st);
   if (err != cudaSuccess) return err;
 
   // router and constant-expert weights: [dG | dz]^T x, rows 0..N-1 -> dW_r, the rest -> dW_c

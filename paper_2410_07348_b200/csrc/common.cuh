@@ -96,6 +96,16 @@ cudaError_t launch_ffn_backward_simt(const Dims& d, const void* x_perm, const in
                                      void* gate_buf, void* up_buf, void* dx_perm, float* dW_gate, float* dW_up,
                                      float* dW_down, cudaStream_t st);
 
+// The same on the tensor cores (bf16, segments of whole 64-row tiles); cudaErrorNotSupported otherwise.
+cudaError_t launch_ffn_backward_tc(const Dims& d, const void* x_perm, const int32_t* offsets, const void* W_gate,
+                                   const void* W_up, const void* W_down, const void* h, const void* dy_perm,
+                                   void* gate_buf, void* up_buf, void* dx_perm, float* dW_gate, float* dW_up,
+                                   float* dW_down, cudaStream_t st);
+
+// C[r, :] = A[r, :] B[e]^T on the forward tensor-core kernel (A [M_cap, Kd], B [n_ffn, Nout, Kd], bf16)
+cudaError_t launch_grouped_gemm_tcgen05(const Dims& d, const void* A, const void* B, void* C, const int32_t* offsets,
+                                        int Nout, int Kd, cudaStream_t st);
+
 // Whole backward pass of one layer; grads are overwritten.
 cudaError_t launch_layer_backward(const Dims& d, const ForwardState& fs, const moepp_weights& w, const void* x,
                                   const float* prev, const void* dy, const float* dlogits_next,

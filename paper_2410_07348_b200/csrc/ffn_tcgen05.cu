@@ -364,6 +364,28 @@ cudaError_t launch_ffn_tcgen05(const Dims& d, const void* x_perm, const int32_t*
   return cudaGetLastError();
 }
 
+// Plain grouped product on the same kernel: C[r, :] = A[r, :] B[e]^T for the rows r of expert e's segment,
+// A [M_cap, Kd], B [n_ffn, Nout, Kd], C [M_cap, Nout], all bf16.
+cudaError_t launch_grouped_gemm_tcgen05(const Dims& d, const void* A, const void* B, void* C, const int32_t* offsets,
+                                        int Nout, int Kd, cudaStream_t st) {
+  if (d.T == 0 || d.n_ffn == 0 || d.M_cap == 0) return cudaSuccess;
+  int dev = 0, sms = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return err;
+  err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (err != cudaSuccess) return err;
+  CUtensorMap mA, mB;
+  if (!make_bf16_tile_map(&mA, A, (uint64_t)d.M_cap, (uint64_t)Kd, BM) ||
+      !make_bf16_tile_map(&mB, B, (uint64_t)d.n_ffn * Nout, (uint64_t)Kd, 256))
+    return cudaErrorNotSupported;
+  auto k2 = grouped_gemm_kernel<false, false>;
+  err = cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  if (err != cudaSuccess) return err;
+  k2<<<sms, kThreads, kSmemBytes, st>>>(mA, mB, mB, static_cast<__nv_bfloat16*>(C), offsets, d.n_ffn, Nout, Kd, nullptr,
+                                        1, 0);
+  return cudaGetLastError();
+}
+
 // The same FFN with GEMM 1 reading its rows straight from x through slot_of_row (no grouped copy of x).
 cudaError_t launch_ffn_tcgen05_gather(const Dims& d, const void* x, const int32_t* slot_of_row, const int32_t* offsets,
                                       const void* W_gate, const void* W_up, const void* W_down, void* h, void* y_perm,

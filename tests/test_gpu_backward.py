@@ -118,3 +118,22 @@ def test_backward_no_tokens():
     got, _ = gpu_backward(cfg, wd, lt.x.cuda(), lt.prev.cuda(), torch.empty(0, 64, device="cuda"), None)
     for name in GRADS[2:]:
         assert not np.any(got[name]), name
+
+
+def test_backward_tensor_core_path_matches_fma_path():
+    """At a size the oracle cannot cover in seconds: the tensor-core GEMMs (row_align 128) against the FMA kernels
+    (forced by flag) on the same forward state; both were checked against the oracle at smaller sizes above."""
+    spec = W.LayerSpec(T=6000, D=1032, F=1416, n_ffn=6, n_zero=1, n_copy=1, n_const=1, top_k=2, dtype="bf16")
+    lt = W.make_layer(spec, seed=5, with_prev=True, w_std=0.03)
+    wd = B.weights_from_tensors(lt)
+    x, prev = lt.x.cuda(), lt.prev.cuda()
+    gen = torch.Generator().manual_seed(9)
+    dy = torch.randn(spec.T, spec.D, generator=gen).to(x.dtype).cuda()
+    res = []
+    for flags in (0, B.FLAG_SIMT_FFN):
+        cfg = B.config_from_spec(spec, row_align=128, flags=flags)
+        res.append(gpu_backward(cfg, wd, x, prev, dy, None)[0])
+    for name in GRADS:
+        a, b = res[0][name], res[1][name]
+        scale = max(float(np.abs(b).max()), 1e-6)
+        assert float(np.abs(a - b).max()) / scale <= 1e-2, name
