@@ -210,6 +210,7 @@ def main():
     ap.add_argument("--tau", type=float, default=1.0, help="Eq. 7 / Eq. 8 weight of the zero-computation experts")
     ap.add_argument("--layers", type=int, default=0, help="use only the first N layers of the workload (profiling)")
     ap.add_argument("--flags", type=int, default=0, help="MOEPP_FLAG_* bits passed in the configuration")
+    ap.add_argument("--no-backward", action="store_true", help="skip the backward-pass timing of layer 1")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "moepp" else args.warmup
 
@@ -343,6 +344,52 @@ def main():
     t_roof_ms = max(flops_ffn / (peaks["burst"] * 1e12), bytes_layer / (peaks["hbm_gbs"] * 1e9)) * 1e3
     layer_ms = ms_step / L
 
+    # ---- backward pass of layer 1: forward with 64-row segments, then moepp_layer_backward ----------------------
+    bwd = None
+    if not args.no_backward:
+        fz = lambda *shape: torch.empty(*shape, device=dev)
+        grads = dict(dx=torch.empty_like(x0), dprev=fz(T, N) if p1 is not None else None, dW_r=fz(N, spec.D),
+                     dW_g=fz(N, N) if p1 is not None else None, dbias=fz(N), dW_c=fz(max(spec.n_const, 1), 2, spec.D),
+                     dv=fz(max(spec.n_const, 1), spec.D), dW_gate=fz(spec.n_ffn, spec.F, spec.D),
+                     dW_up=fz(spec.n_ffn, spec.F, spec.D), dW_down=fz(spec.n_ffn, spec.D, spec.F))
+        dy = torch.randn(T, spec.D, device=dev).to(td)
+        reps_b = max(5, args.steps // 5)
+
+        def fwd_bwd(flags, gemm_units):
+            cfg_b = B.config_from_spec(spec, add_residual=add_res, flags=flags, tau=args.tau,
+                                       capacity_factor=args.capacity_factor, row_align=64)
+            ws_f = torch.empty(B.moepp_workspace_bytes(cfg_b), dtype=torch.uint8, device=dev)
+            ws_b = torch.empty(B.moepp_backward_workspace_bytes(cfg_b), dtype=torch.uint8, device=dev)
+            pair = [("forward", lambda: B.moepp_layer_forward(cfg_b, wd, x0, p1, yb, lgs[0], ws_f)),
+                    ("backward", lambda: B.moepp_layer_backward(cfg_b, wd, x0, p1, lgs[0], dy, None, ws_f, grads, ws_b))]
+            acc_b = {n: 0.0 for n, _ in pair}
+            for it in range(3 + reps_b):
+                evs = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+                evs[0].record()
+                for i, (_, fn) in enumerate(pair):
+                    fn()
+                    evs[i + 1].record()
+                torch.cuda.synchronize()
+                if it >= 3:
+                    for i, (n, _) in enumerate(pair):
+                        acc_b[n] += evs[i].elapsed_time(evs[i + 1]) / reps_b
+            assert B.moepp_device_error() == 0
+            B.moepp_route(cfg_b, x0, wd["W_r"], wd["W_g"], p1, wd["router_bias"], None, lgs[0], idx, wk, cnt, off, None)
+            M_b = int(off[-1].item())
+            flops_b = gemm_units * spec.D * spec.F * M_b
+            t_roof_b = flops_b / (peaks["burst"] * 1e12) * 1e3
+            return {"ms_forward": acc_b["forward"], "ms_backward": acc_b["backward"], "ffn_rows": M_b,
+                    "ffn_flops_backward": flops_b, "t_roof_ms": t_roof_b, "frac": t_roof_b / acc_b["backward"],
+                    "tflops_whole_backward": flops_b / (acc_b["backward"] * 1e-3) / 1e12,
+                    "tokens_per_s_fwd_bwd": world * T / ((acc_b["forward"] + acc_b["backward"]) * 1e-3)}
+
+        # dH 2, dXp 4, three weight gradients 6 (x M D F); recomputing gate and up adds 4
+        bwd = {"what": "layer 1, segments padded to 64 rows; backward = moepp_layer_backward (all gradients); "
+                       "roofline = FFN GEMM flops of the pass at the bf16 burst peak",
+               "kept_pre_activations": fwd_bwd(args.flags | B.FLAG_SAVE_PREACT, 12.0),
+               "recomputed_pre_activations": fwd_bwd(args.flags, 16.0)}
+        del grads
+
     # ---- end to end through the host-buffer call --------------------------------------------------------------
     xh = x0.cpu().pin_memory()
     yh = torch.empty(T, spec.D, dtype=td).pin_memory()
@@ -396,6 +443,7 @@ def main():
         "vanilla": {"value": world * tokens_per_step / (ms_van * 1e-3), "unit": UNIT, "ms_per_step": ms_van,
                     "speedup_of_moepp": ms_van / ms_step,
                     "what": "same library, same T, D, F, n_ffn, K, no zero-computation experts"},
+        "backward": bwd,
         "cpu_baseline": cpu,
         "paper_context": "paper reports 1.1-2.1x expert forward throughput over vanilla MoE (A100 cluster, conditions "
                          "unstated); context only",

@@ -63,6 +63,9 @@ typedef enum { MOEPP_F32 = 0, MOEPP_BF16 = 1 } moepp_dtype;
 #define MOEPP_FLAG_FUSED_GATHER 8  /* moepp_layer_forward, bf16: GEMM 1 fetches its rows from x with TMA gather loads
                                       and x_perm is never built (measured slower than the staged default on B200) */
 #define MOEPP_FLAG_FFN_SINGLE_CTA 4 /* bf16 only: 128x256 tiles on single CTAs instead of 256x256 on CTA pairs */
+#define MOEPP_FLAG_SAVE_PREACT 16 /* moepp_layer_forward: also keep the SwiGLU pre-activations (gate and up, [M_cap, F]
+                                     each) in the workspace, which grows accordingly; moepp_layer_backward then skips
+                                     their recomputation.  Not with MOEPP_FLAG_FFN_SINGLE_CTA / MOEPP_FLAG_FUSED_GATHER. */
 
 typedef struct {
   int32_t T, D, F;
@@ -247,7 +250,10 @@ moepp_status moepp_backward_workspace_bytes(const moepp_config* cfg, size_t* byt
  * nothing, Eq. 4 passes w dy to x, Eq. 5 also feeds dv and the two mixing logits), gate backward (softmax
  * over all N, renormalisation if on), the expert FFNs (SwiGLU pre-activations recomputed from x_perm),
  * the router (dW_r, dW_g, dbias, dprev) and dx.  Slots dropped by Eq. 8 carry no gradient.
- * The FFN GEMMs of this pass run on the FMA units (float accumulation) for both dtypes.
+ * bf16 with row_align a multiple of 64: the FFN GEMMs run on the tensor cores, operands read in place (the
+ * transposed products take their tiles MN-major); otherwise on the FMA units.  Float accumulation either way.
+ * With MOEPP_FLAG_SAVE_PREACT (set in the forward call too) the pre-activations are read from fwd_workspace
+ * instead of being recomputed.
  * MOEPP_FLAG_FUSED_GATHER is refused (that forward path does not keep x_perm).
  * Errors: as moepp_layer_forward; MOEPP_ERR_WORKSPACE when either workspace is too small.
  */

@@ -54,6 +54,7 @@ inline moepp_status from_cuda(cudaError_t e) { return e == cudaSuccess ? MOEPP_O
 // Regions of the layer workspace, in order.  `host_io` adds device staging for x, prev, y.
 struct Carve {
   size_t logits, topk_idx, topk_w, counts, offsets, alpha, row_of_slot, slot_of_row, x_perm, h, y_perm;
+  size_t gate, up;  // SwiGLU pre-activations, only with MOEPP_FLAG_SAVE_PREACT
   size_t x_dev, prev_dev, y_dev;
   size_t total;
 };
@@ -79,6 +80,10 @@ Carve carve(const Dims& d, bool host_io) {
   c.x_perm = take(es * (size_t)d.M_cap * d.D);
   c.h = take(es * (size_t)d.M_cap * d.F);
   c.y_perm = take(es * (size_t)d.M_cap * d.D);
+  if (d.flags & MOEPP_FLAG_SAVE_PREACT) {
+    c.gate = take(es * (size_t)d.M_cap * d.F);
+    c.up = take(es * (size_t)d.M_cap * d.F);
+  }
   if (host_io) {
     c.x_dev = take(es * (size_t)d.T * d.D);
     c.prev_dev = take(sizeof(float) * (size_t)d.T * d.N);
@@ -89,15 +94,18 @@ Carve carve(const Dims& d, bool host_io) {
 }
 
 moepp_status ffn_dispatch(const Dims& d, const void* x_perm, const int32_t* offsets, const void* W_gate,
-                          const void* W_up, const void* W_down, void* h, void* y_perm, cudaStream_t st) {
+                          const void* W_up, const void* W_down, void* h, void* y_perm, cudaStream_t st,
+                          void* gate_out = nullptr, void* up_out = nullptr) {
   if (d.n_ffn == 0 || d.T == 0) return MOEPP_OK;
   if (d.dtype == MOEPP_BF16 && !(d.flags & MOEPP_FLAG_SIMT_FFN)) {
-    const cudaError_t e = ((d.flags & MOEPP_FLAG_FFN_SINGLE_CTA) ? launch_ffn_tcgen05 : launch_ffn_tcgen05_pair)(
-        d, x_perm, offsets, W_gate, W_up, W_down, h, y_perm, st);
+    const cudaError_t e =
+        (d.flags & MOEPP_FLAG_FFN_SINGLE_CTA)
+            ? launch_ffn_tcgen05(d, x_perm, offsets, W_gate, W_up, W_down, h, y_perm, st)
+            : launch_ffn_tcgen05_pair(d, x_perm, offsets, W_gate, W_up, W_down, h, y_perm, st, gate_out, up_out);
     // a shape the TMA tensor maps cannot describe runs on the FMA kernels instead
     if (e != cudaErrorNotSupported) return from_cuda(e);
   }
-  return from_cuda(launch_ffn_simt(d, x_perm, offsets, W_gate, W_up, W_down, h, y_perm, st));
+  return from_cuda(launch_ffn_simt(d, x_perm, offsets, W_gate, W_up, W_down, h, y_perm, st, gate_out, up_out));
 }
 
 moepp_status layer_on_device(const Dims& d, const Carve& c, const moepp_weights* w, const void* x,
@@ -128,7 +136,9 @@ moepp_status layer_on_device(const Dims& d, const Carve& c, const moepp_weights*
       if (e != cudaSuccess) return MOEPP_ERR_CUDA;
     }
   } else {
-    const moepp_status s = ffn_dispatch(d, x_perm, offsets, w->W_gate, w->W_up, w->W_down, h, y_perm, st);
+    const bool keep = (d.flags & MOEPP_FLAG_SAVE_PREACT) != 0;
+    const moepp_status s = ffn_dispatch(d, x_perm, offsets, w->W_gate, w->W_up, w->W_down, h, y_perm, st,
+                                        keep ? ws + c.gate : nullptr, keep ? ws + c.up : nullptr);
     if (s != MOEPP_OK) return s;
   }
   e = launch_combine(d, x, y_perm, topk_idx, topk_w, row_of_slot, alpha, w->W_c, w->v, y, st);
@@ -140,6 +150,8 @@ moepp_status check_layer_args(const Dims& d, const moepp_weights* w, const void*
   if (w == nullptr || ws == nullptr) return MOEPP_ERR_INVALID_ARG;
   if (d.T > 0 && (x == nullptr || y == nullptr)) return MOEPP_ERR_INVALID_ARG;
   if (d.flags & MOEPP_FLAG_LOGITS_GIVEN) return MOEPP_ERR_INVALID_ARG;  // a whole layer computes its own logits
+  if ((d.flags & MOEPP_FLAG_SAVE_PREACT) && (d.flags & (MOEPP_FLAG_FFN_SINGLE_CTA | MOEPP_FLAG_FUSED_GATHER)))
+    return MOEPP_ERR_INVALID_ARG;  // only the default and the FMA kernels store the pre-activations
   if (w->W_r == nullptr) return MOEPP_ERR_INVALID_ARG;
   if (d.T > 0 && (w->W_g == nullptr) != (prev == nullptr)) return MOEPP_ERR_INVALID_ARG;
   if (d.n_const > 0 && (w->W_c == nullptr || w->v == nullptr)) return MOEPP_ERR_INVALID_ARG;
@@ -607,6 +619,9 @@ moepp_status moepp_layer_backward(const moepp_config* cfg, const moepp_weights* 
   fs.x_perm = fw + c.x_perm;
   fs.h = fw + c.h;
   fs.y_perm = fw + c.y_perm;
+  const bool kept = (d.flags & MOEPP_FLAG_SAVE_PREACT) != 0;
+  fs.gate = kept ? fw + c.gate : nullptr;
+  fs.up = kept ? fw + c.up : nullptr;
   BackwardScratch b{};
   b.dYp = bw + bc.dYp; b.gate = bw + bc.gate; b.up = bw + bc.up; b.dXp = bw + bc.dXp;
   b.dw = reinterpret_cast<float*>(bw + bc.dw);

@@ -269,51 +269,139 @@ __global__ void __launch_bounds__(256) column_sum_kernel(const float* __restrict
   if (threadIdx.x == 0) out[blockIdx.x] = s[0];
 }
 
-// One warp per token: dx = cx dy + sum_r dGz[t, r] Wrow_r + sum over kept FFN picks of dXp[row_k, :],
+constexpr int kDxTokens = 8;  // tokens per warp in dx_assemble
+
+// dx = cx dy + sum_r dGz[t, r] Wrow_r + sum over kept FFN picks of dXp[row_k, :],
 // Wrow_r = W_r[r, :] for r < N and the flattened W_c rows after that.
+// One warp owns kDxTokens tokens and walks the columns 256 at a time (8 per lane), so that every weight row it
+// reads is used for all its tokens.
 template <typename XT>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 dx_assemble_kernel(Dims dm, int R, const XT* __restrict__ dy, const float* __restrict__ cx,
                    const float* __restrict__ dGz, const float* __restrict__ W_r, const float* __restrict__ W_c,
                    const XT* __restrict__ dXp, const int32_t* __restrict__ topk_idx,
                    const int32_t* __restrict__ row_of_slot, XT* __restrict__ dx) {
-  __shared__ float s_c[kWarpsPerBlock][kMaxRouteRows];
+  extern __shared__ float s_dx[];  // per warp: [R][kDxTokens] coefficients, then [kDxTokens] cx, then rows
   const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
-  const long long t = (long long)blockIdx.x * kWarpsPerBlock + wib;
-  if (t >= dm.T) return;
   const int D = dm.D, N = dm.N, K = dm.K;
-  for (int r = lane; r < R; r += 32) s_c[wib][r] = dGz[t * R + r];
-  int rows[kMaxTopK];
-#pragma unroll
-  for (int k = 0; k < kMaxTopK; ++k) {
-    rows[k] = -1;
-    if (k < K && topk_idx[t * K + k] < dm.n_ffn) rows[k] = row_of_slot[t * K + k];  // -2 when dropped
+  const int per_warp = R * kDxTokens + kDxTokens + kDxTokens * kMaxTopK;
+  float* s_c = s_dx + (size_t)wib * per_warp;
+  float* s_cx = s_c + R * kDxTokens;
+  int* s_rows = reinterpret_cast<int*>(s_cx + kDxTokens);
+  const long long t0 = ((long long)blockIdx.x * kWarpsPerBlock + wib) * kDxTokens;
+  if (t0 >= dm.T) return;
+  const int nt = (int)min((long long)kDxTokens, dm.T - t0);
+  for (int i = lane; i < R * kDxTokens; i += 32) {
+    const int r = i / kDxTokens, j = i % kDxTokens;
+    s_c[i] = j < nt ? dGz[(t0 + j) * R + r] : 0.f;
   }
+  for (int i = lane; i < kDxTokens * kMaxTopK; i += 32) {
+    const int j = i / kMaxTopK, k = i % kMaxTopK;
+    int row = -1;
+    if (j < nt && k < K && topk_idx[(t0 + j) * K + k] < dm.n_ffn) row = row_of_slot[(t0 + j) * K + k];  // -2: dropped
+    s_rows[i] = row;
+  }
+  if (lane < kDxTokens) s_cx[lane] = lane < nt ? cx[t0 + lane] : 0.f;
   __syncwarp();
-  const float c = cx[t];
   for (int d = lane * 8; d < D; d += 256) {
-    float acc[8], tmp[8];
-    Vec8<XT>::load(dy + (size_t)t * D + d, tmp);
+    float acc[kDxTokens][8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) acc[i] = c * tmp[i];
+    for (int j = 0; j < kDxTokens; ++j)
+#pragma unroll
+      for (int i = 0; i < 8; ++i) acc[j][i] = 0.f;
     for (int r = 0; r < R; ++r) {
-      const float g = s_c[wib][r];
       const float* wrow = r < N ? W_r + (size_t)r * D + d : W_c + (size_t)(r - N) * D + d;
       const float4 a = __ldg(reinterpret_cast<const float4*>(wrow));
       const float4 b = __ldg(reinterpret_cast<const float4*>(wrow + 4));
-      acc[0] = fmaf(g, a.x, acc[0]); acc[1] = fmaf(g, a.y, acc[1]); acc[2] = fmaf(g, a.z, acc[2]);
-      acc[3] = fmaf(g, a.w, acc[3]); acc[4] = fmaf(g, b.x, acc[4]); acc[5] = fmaf(g, b.y, acc[5]);
-      acc[6] = fmaf(g, b.z, acc[6]); acc[7] = fmaf(g, b.w, acc[7]);
+      const float wv[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+      const float4 c0 = *reinterpret_cast<const float4*>(s_c + r * kDxTokens);
+      const float4 c1 = *reinterpret_cast<const float4*>(s_c + r * kDxTokens + 4);
+      const float cj[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+#pragma unroll
+      for (int j = 0; j < kDxTokens; ++j)
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[j][i] = fmaf(cj[j], wv[i], acc[j][i]);
     }
 #pragma unroll
-    for (int k = 0; k < kMaxTopK; ++k) {
-      if (rows[k] >= 0) {
-        Vec8<XT>::load(dXp + (size_t)rows[k] * D + d, tmp);
+    for (int j = 0; j < kDxTokens; ++j) {
+      if (j < nt) {
+        float tmp[8];
+        const float c = s_cx[j];
+        Vec8<XT>::load(dy + (size_t)(t0 + j) * D + d, tmp);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) acc[i] += tmp[i];
+        for (int i = 0; i < 8; ++i) acc[j][i] = fmaf(c, tmp[i], acc[j][i]);
+        for (int k = 0; k < K; ++k) {
+          const int row = s_rows[j * kMaxTopK + k];
+          if (row >= 0) {
+            Vec8<XT>::load(dXp + (size_t)row * D + d, tmp);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) acc[j][i] += tmp[i];
+          }
+        }
+        Vec8<XT>::store(dx + (size_t)(t0 + j) * D + d, acc[j]);
       }
     }
-    Vec8<XT>::store(dx + (size_t)t * D + d, acc);
+  }
+}
+
+constexpr int kRt = 12;  // rows of the small factor per pass in token_outer_rows
+
+// part[z, m, n] = sum over the tokens t of chunk z of A[t, m] * B[t, n] for a SMALL M (a few dozen rows) and a wide,
+// 8-aligned Nout: each thread keeps kRt x 4 sums for 4 columns, the block covers 1024 columns, and the rows of A
+// are taken kRt at a time (the chunk of B is read again from cache for each group).
+template <typename TB>
+__global__ void __launch_bounds__(256)
+token_outer_rows_kernel(const float* __restrict__ A, const TB* __restrict__ B, float* __restrict__ part, int T, int M,
+                        int Nout, long long a_rs, long long b_rs, int chunk) {
+  constexpr int TS = 32;  // tokens staged per trip
+  __shared__ __align__(16) float s_a[TS][kRt];
+  const int z = blockIdx.y, n = (blockIdx.x * 256 + threadIdx.x) * 4;
+  const int t_begin = z * chunk, t_end = min(T, t_begin + chunk);
+  const bool col_ok = n < Nout;  // Nout is a multiple of 4
+  for (int m0 = 0; m0 < M; m0 += kRt) {
+    float acc[kRt][4];
+#pragma unroll
+    for (int r = 0; r < kRt; ++r) acc[r][0] = acc[r][1] = acc[r][2] = acc[r][3] = 0.f;
+    for (int ts = t_begin; ts < t_end; ts += TS) {
+      __syncthreads();
+      for (int i = threadIdx.x; i < TS * kRt; i += 256) {
+        const int tt = i / kRt, r = i % kRt;
+        s_a[tt][r] = (ts + tt < t_end && m0 + r < M) ? A[(size_t)(ts + tt) * a_rs + m0 + r] : 0.f;
+      }
+      __syncthreads();
+      if (col_ok) {
+#pragma unroll 4
+        for (int tt = 0; tt < TS; ++tt) {
+          float bv[4] = {0.f, 0.f, 0.f, 0.f};
+          if (ts + tt < t_end) {
+            const TB* bp = B + (size_t)(ts + tt) * b_rs + n;
+            if (sizeof(TB) == 2) {
+              const uint2 u = *reinterpret_cast<const uint2*>(bp);
+              bv[0] = bf16_lo(u.x); bv[1] = bf16_hi(u.x); bv[2] = bf16_lo(u.y); bv[3] = bf16_hi(u.y);
+            } else {
+              const float4 f = *reinterpret_cast<const float4*>(bp);
+              bv[0] = f.x; bv[1] = f.y; bv[2] = f.z; bv[3] = f.w;
+            }
+          }
+#pragma unroll
+          for (int r4 = 0; r4 < kRt; r4 += 4) {
+            const float4 av = *reinterpret_cast<const float4*>(&s_a[tt][r4]);
+            const float ar[4] = {av.x, av.y, av.z, av.w};
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+#pragma unroll
+              for (int i = 0; i < 4; ++i) acc[r4 + r][i] = fmaf(ar[r], bv[i], acc[r4 + r][i]);
+          }
+        }
+      }
+    }
+    if (col_ok) {
+#pragma unroll
+      for (int r = 0; r < kRt; ++r)
+        if (m0 + r < M)
+          *reinterpret_cast<float4*>(part + ((size_t)z * M + m0 + r) * Nout + n) =
+              make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
+    }
   }
 }
 
@@ -336,8 +424,13 @@ cudaError_t token_outer(const Dims& d, const float* A, long long a_rs, int M, co
   if (M == 0 || Nout == 0) return cudaSuccess;
   int chunk;
   const int Z = backward_token_chunks(d, &chunk);
-  dim3 grid((unsigned)((M + kOm - 1) / kOm), (unsigned)((Nout + kOn - 1) / kOn), (unsigned)Z);
-  token_outer_kernel<TB><<<grid, 256, 0, st>>>(A, B, part, d.T, M, Nout, a_rs, b_rs, chunk);
+  if (Nout % 8 == 0 && Nout >= 256 && b_rs % 8 == 0) {
+    dim3 grid((unsigned)((Nout + 1023) / 1024), (unsigned)Z);
+    token_outer_rows_kernel<TB><<<grid, 256, 0, st>>>(A, B, part, d.T, M, Nout, a_rs, b_rs, chunk);
+  } else {
+    dim3 grid((unsigned)((M + kOm - 1) / kOm), (unsigned)((Nout + kOn - 1) / kOn), (unsigned)Z);
+    token_outer_kernel<TB><<<grid, 256, 0, st>>>(A, B, part, d.T, M, Nout, a_rs, b_rs, chunk);
+  }
   cudaError_t err = cudaGetLastError();
   if (err != cudaSuccess) return err;
   const long long n = (long long)M * Nout;
@@ -369,10 +462,10 @@ cudaError_t layer_backward_t(const Dims& d, const ForwardState& fs, const moepp_
   err = cudaErrorNotSupported;
   if (!(d.flags & MOEPP_FLAG_SIMT_FFN))
     err = launch_ffn_backward_tc(d, fs.x_perm, fs.offsets, w.W_gate, w.W_up, w.W_down, fs.h, b.dYp, b.gate, b.up,
-                                 b.dXp, g.dW_gate, g.dW_up, g.dW_down, st);
+                                 b.dXp, g.dW_gate, g.dW_up, g.dW_down, st, fs.gate, fs.up);
   if (err == cudaErrorNotSupported)
     err = launch_ffn_backward_simt(d, fs.x_perm, fs.offsets, w.W_gate, w.W_up, w.W_down, fs.h, b.dYp, b.gate, b.up,
-                                   b.dXp, g.dW_gate, g.dW_up, g.dW_down, st);
+                                   b.dXp, g.dW_gate, g.dW_up, g.dW_down, st, fs.gate, fs.up);
   if (err != cudaSuccess) return err;
 
   // router and constant-expert weights: [dG | dz]^T x, rows 0..N-1 -> dW_r, the rest -> dW_c
@@ -391,7 +484,13 @@ cudaError_t layer_backward_t(const Dims& d, const ForwardState& fs, const moepp_
     column_sum_kernel<<<(unsigned)d.N, 256, 0, st>>>(b.dGz, g.dbias, d.T, R);
     if ((err = cudaGetLastError()) != cudaSuccess) return err;
   }
-  dx_assemble_kernel<XT><<<token_blocks, kWarpsPerBlock * 32, 0, st>>>(
+  const unsigned dx_blocks = (unsigned)((d.T + kWarpsPerBlock * kDxTokens - 1) / (kWarpsPerBlock * kDxTokens));
+  const size_t dx_smem = sizeof(float) * kWarpsPerBlock * ((size_t)R * kDxTokens + kDxTokens + kDxTokens * kMaxTopK);
+  if (dx_smem > 48 * 1024) {
+    err = cudaFuncSetAttribute(dx_assemble_kernel<XT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dx_smem);
+    if (err != cudaSuccess) return err;
+  }
+  dx_assemble_kernel<XT><<<dx_blocks, kWarpsPerBlock * 32, dx_smem, st>>>(
       d, R, dy, b.cx, b.dGz, w.W_r, w.W_c, static_cast<const XT*>(b.dXp), fs.topk_idx, fs.row_of_slot,
       static_cast<XT*>(g.dx));
   return cudaGetLastError();

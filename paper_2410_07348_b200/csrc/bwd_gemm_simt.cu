@@ -19,7 +19,8 @@ __device__ __forceinline__ void stf(__nv_bfloat16* p, float v) { *p = __float2bf
 struct RowsArgs {
   const void *A, *B, *A2, *B2;   // second product optional (A2 == nullptr)
   void* C;
-  void *gate, *up;               // SwiGLU-backward epilogue: pre-activations in, dGate / dUp out (C unused)
+  void *gate, *up;               // SwiGLU-backward epilogue: dGate / dUp out (C unused)
+  const void *gate_in, *up_in;   // ... and the pre-activations it reads (may be the same buffers)
   const int32_t* offsets;
   int n_ffn, Nout, Kd;
   long long a_rs, c_rs;          // row strides of A (and A2) and C
@@ -84,7 +85,8 @@ __global__ void __launch_bounds__(256) bwd_rows_kernel(RowsArgs a) {
       } else {
         T* gp = static_cast<T*>(a.gate) + at;
         T* up = static_cast<T*>(a.up) + at;
-        const float g = ldf(gp), u = ldf(up), s = 1.f / (1.f + expf(-g)), dh = acc[i][j];
+        const float g = ldf(static_cast<const T*>(a.gate_in) + at), u = ldf(static_cast<const T*>(a.up_in) + at);
+        const float s = 1.f / (1.f + expf(-g)), dh = acc[i][j];
         stf(gp, dh * u * (s + g * s * (1.f - s)));
         stf(up, dh * g * s);
       }
@@ -149,17 +151,21 @@ template <typename T>
 cudaError_t ffn_backward_t(const Dims& d, const void* x_perm, const int32_t* offsets, const void* W_gate,
                            const void* W_up, const void* W_down, const void* h, const void* dy_perm, void* gate_buf,
                            void* up_buf, void* dx_perm, float* dW_gate, float* dW_up, float* dW_down,
-                           cudaStream_t st) {
+                           cudaStream_t st, const void* gate_in, const void* up_in) {
   const long long D = d.D, F = d.F;
   cudaError_t err;
-  RowsArgs a{};
-  a.offsets = offsets; a.n_ffn = d.n_ffn;
-  // 1-2. SwiGLU pre-activations again: gate = Xp W_gate^T, up = Xp W_up^T
-  a.A = x_perm; a.a_rs = D; a.Kd = d.D; a.Nout = d.F; a.c_rs = F; a.b_es = F * D; a.b_ks = 1; a.b_ns = D;
-  a.B = W_gate; a.C = gate_buf;
-  if ((err = run_rows<T>(d, a, false, st)) != cudaSuccess) return err;
-  a.B = W_up; a.C = up_buf;
-  if ((err = run_rows<T>(d, a, false, st)) != cudaSuccess) return err;
+  if (gate_in == nullptr) {
+    // 1-2. SwiGLU pre-activations again: gate = Xp W_gate^T, up = Xp W_up^T
+    RowsArgs a{};
+    a.offsets = offsets; a.n_ffn = d.n_ffn;
+    a.A = x_perm; a.a_rs = D; a.Kd = d.D; a.Nout = d.F; a.c_rs = F; a.b_es = F * D; a.b_ks = 1; a.b_ns = D;
+    a.B = W_gate; a.C = gate_buf;
+    if ((err = run_rows<T>(d, a, false, st)) != cudaSuccess) return err;
+    a.B = W_up; a.C = up_buf;
+    if ((err = run_rows<T>(d, a, false, st)) != cudaSuccess) return err;
+    gate_in = gate_buf;
+    up_in = up_buf;
+  }
   // 3. dW_down[e] = dYp_e^T H_e
   dim3 gdn((unsigned)((d.D + TM - 1) / TM), (unsigned)((d.F + TN - 1) / TN), (unsigned)d.n_ffn);
   bwd_wgrad_kernel<T><<<gdn, 256, 0, st>>>(static_cast<const T*>(dy_perm), static_cast<const T*>(h), dW_down, offsets,
@@ -169,7 +175,7 @@ cudaError_t ffn_backward_t(const Dims& d, const void* x_perm, const int32_t* off
   RowsArgs b{};
   b.offsets = offsets; b.n_ffn = d.n_ffn;
   b.A = dy_perm; b.a_rs = D; b.Kd = d.D; b.Nout = d.F; b.c_rs = F; b.B = W_down; b.b_es = D * F; b.b_ks = F; b.b_ns = 1;
-  b.gate = gate_buf; b.up = up_buf;
+  b.gate = gate_buf; b.up = up_buf; b.gate_in = gate_in; b.up_in = up_in;
   if ((err = run_rows<T>(d, b, true, st)) != cudaSuccess) return err;
   // 5. dW_gate[e] = dGate_e^T Xp_e, dW_up[e] = dUp_e^T Xp_e
   dim3 gup((unsigned)((d.F + TM - 1) / TM), (unsigned)((d.D + TN - 1) / TN), (unsigned)d.n_ffn);
@@ -194,7 +200,7 @@ cudaError_t ffn_backward_t(const Dims& d, const void* x_perm, const int32_t* off
 cudaError_t launch_ffn_backward_simt(const Dims& d, const void* x_perm, const int32_t* offsets, const void* W_gate,
                                      const void* W_up, const void* W_down, const void* h, const void* dy_perm,
                                      void* gate_buf, void* up_buf, void* dx_perm, float* dW_gate, float* dW_up,
-                                     float* dW_down, cudaStream_t st) {
+                                     float* dW_down, cudaStream_t st, const void* gate_in, const void* up_in) {
   if (d.n_ffn == 0) return cudaSuccess;
   const size_t wbytes = sizeof(float) * (size_t)d.n_ffn * d.D * d.F;
   cudaError_t err;  // experts without rows still get a defined (zero) gradient
@@ -205,9 +211,9 @@ cudaError_t launch_ffn_backward_simt(const Dims& d, const void* x_perm, const in
   }
   return d.dtype == MOEPP_BF16
              ? ffn_backward_t<__nv_bfloat16>(d, x_perm, offsets, W_gate, W_up, W_down, h, dy_perm, gate_buf, up_buf,
-                                             dx_perm, dW_gate, dW_up, dW_down, st)
+                                             dx_perm, dW_gate, dW_up, dW_down, st, gate_in, up_in)
              : ffn_backward_t<float>(d, x_perm, offsets, W_gate, W_up, W_down, h, dy_perm, gate_buf, up_buf, dx_perm,
-                                     dW_gate, dW_up, dW_down, st);
+                                     dW_gate, dW_up, dW_down, st, gate_in, up_in);
 }
 
 }  // namespace moepp

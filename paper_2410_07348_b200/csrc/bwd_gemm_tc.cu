@@ -52,7 +52,8 @@ struct TileInfo {
 
 struct Args {
   void* C;                 // DX: bf16 [M_cap, Nout];  WGRAD: float [n_ffn, Mout, Nout]
-  __nv_bfloat16 *gate, *up;  // DH
+  __nv_bfloat16 *gate, *up;  // DH: dGate, dUp out
+  const __nv_bfloat16 *gate_in, *up_in;  // DH: pre-activations in (may be the same buffers)
   const int32_t* offsets;
   int n_ffn, Mout, Nout, Kd;
   int32_t* err_word;
@@ -269,8 +270,8 @@ bwd_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant_
               __nv_bfloat16* gp = a.gate + at + c + 8 * half;
               __nv_bfloat16* up = a.up + at + c + 8 * half;
               float g[8], u[8], dg[8], du[8];
-              Vec8<__nv_bfloat16>::load(gp, g);
-              Vec8<__nv_bfloat16>::load(up, u);
+              Vec8<__nv_bfloat16>::load(a.gate_in + at + c + 8 * half, g);
+              Vec8<__nv_bfloat16>::load(a.up_in + at + c + 8 * half, u);
 #pragma unroll
               for (int i = 0; i < 8; ++i) {
                 const float s = 1.f / (1.f + __expf(-g[i]));
@@ -321,7 +322,7 @@ cudaError_t run(int sms, const CUtensorMap& a0, const CUtensorMap& a1, const CUt
 cudaError_t launch_ffn_backward_tc(const Dims& d, const void* x_perm, const int32_t* offsets, const void* W_gate,
                                    const void* W_up, const void* W_down, const void* h, const void* dy_perm,
                                    void* gate_buf, void* up_buf, void* dx_perm, float* dW_gate, float* dW_up,
-                                   float* dW_down, cudaStream_t st) {
+                                   float* dW_down, cudaStream_t st, const void* gate_in, const void* up_in) {
   if (d.dtype != MOEPP_BF16 || d.row_align % 64 != 0) return cudaErrorNotSupported;
   if (d.T == 0 || d.n_ffn == 0 || d.M_cap == 0) return cudaErrorNotSupported;
   int dev = 0, sms = 0;
@@ -347,9 +348,13 @@ cudaError_t launch_ffn_backward_tc(const Dims& d, const void* x_perm, const int3
       !make_bf16_tile_map(&mWuMN, W_up, E * F, D, 64))
     return cudaErrorNotSupported;
 
-  // 1. the SwiGLU pre-activations again: gate = Xp W_gate^T, up = Xp W_up^T
-  if ((err = launch_grouped_gemm_tcgen05(d, x_perm, W_gate, gate_buf, offsets, d.F, d.D, st)) != cudaSuccess) return err;
-  if ((err = launch_grouped_gemm_tcgen05(d, x_perm, W_up, up_buf, offsets, d.F, d.D, st)) != cudaSuccess) return err;
+  // 1. the SwiGLU pre-activations again, unless the forward pass kept them: gate = Xp W_gate^T, up = Xp W_up^T
+  if (gate_in == nullptr) {
+    if ((err = launch_grouped_gemm_tcgen05(d, x_perm, W_gate, gate_buf, offsets, d.F, d.D, st)) != cudaSuccess) return err;
+    if ((err = launch_grouped_gemm_tcgen05(d, x_perm, W_up, up_buf, offsets, d.F, d.D, st)) != cudaSuccess) return err;
+    gate_in = gate_buf;
+    up_in = up_buf;
+  }
 
   Args a{};
   a.offsets = offsets; a.n_ffn = d.n_ffn; a.err_word = err_word;
@@ -358,6 +363,7 @@ cudaError_t launch_ffn_backward_tc(const Dims& d, const void* x_perm, const int3
   if ((err = run<WGRAD>(sms, mDyMN, mDyMN, mHMN, mHMN, a, st)) != cudaSuccess) return err;
   // 3. dH = dYp W_down -> dGate, dUp in place
   a.C = nullptr; a.gate = static_cast<__nv_bfloat16*>(gate_buf); a.up = static_cast<__nv_bfloat16*>(up_buf);
+  a.gate_in = static_cast<const __nv_bfloat16*>(gate_in); a.up_in = static_cast<const __nv_bfloat16*>(up_in);
   a.Mout = 0; a.Nout = d.F; a.Kd = d.D;
   if ((err = run<DH>(sms, mDyK, mDyK, mWdMN, mWdMN, a, st)) != cudaSuccess) return err;
   // 4. dW_gate[e] = dGate_e^T Xp_e, dW_up[e] = dUp_e^T Xp_e

@@ -41,8 +41,10 @@ cudaError_t launch_route_tc(const Dims& d, const void* x, const float* W_r, cons
 cudaError_t launch_permute(const Dims& d, const void* x, const int32_t* topk_idx, const int32_t* offsets,
                            int32_t* row_of_slot, int32_t* slot_of_row, void* x_perm, cudaStream_t st);
 
+// gate_out / up_out (both or neither): the SwiGLU pre-activations [M_cap, F] are stored as well
 cudaError_t launch_ffn_simt(const Dims& d, const void* x_perm, const int32_t* offsets, const void* W_gate,
-                            const void* W_up, const void* W_down, void* h, void* y_perm, cudaStream_t st);
+                            const void* W_up, const void* W_down, void* h, void* y_perm, cudaStream_t st,
+                            void* gate_out = nullptr, void* up_out = nullptr);
 
 // bf16 tensor-core path; returns cudaErrorNotSupported if the tensor maps cannot be encoded.
 cudaError_t launch_ffn_tcgen05(const Dims& d, const void* x_perm, const int32_t* offsets, const void* W_gate,
@@ -55,7 +57,8 @@ cudaError_t launch_ffn_tcgen05_gather(const Dims& d, const void* x, const int32_
 
 // the same on CTA pairs (cta_group::2, 256 x 256 tiles)
 cudaError_t launch_ffn_tcgen05_pair(const Dims& d, const void* x_perm, const int32_t* offsets, const void* W_gate,
-                                    const void* W_up, const void* W_down, void* h, void* y_perm, cudaStream_t st);
+                                    const void* W_up, const void* W_down, void* h, void* y_perm, cudaStream_t st,
+                                    void* gate_out = nullptr, void* up_out = nullptr);
 
 cudaError_t launch_balance_stats(const Dims& d, const float* logits, const int32_t* counts, float* f, float* P,
                                  float* loss, cudaStream_t st);
@@ -77,6 +80,8 @@ struct ForwardState {
   const void* x_perm;
   const void* h;
   const void* y_perm;
+  const void* gate;  // SwiGLU pre-activations [M_cap, F] if the forward pass kept them, else nullptr
+  const void* up;
 };
 
 // Device scratch of one backward pass.
@@ -91,16 +96,19 @@ struct BackwardScratch {
 
 int backward_token_chunks(const Dims& d, int* chunk_tokens);
 
+// gate_in / up_in: pre-activations kept by the forward pass (nullptr: they are recomputed into gate_buf / up_buf)
 cudaError_t launch_ffn_backward_simt(const Dims& d, const void* x_perm, const int32_t* offsets, const void* W_gate,
                                      const void* W_up, const void* W_down, const void* h, const void* dy_perm,
                                      void* gate_buf, void* up_buf, void* dx_perm, float* dW_gate, float* dW_up,
-                                     float* dW_down, cudaStream_t st);
+                                     float* dW_down, cudaStream_t st, const void* gate_in = nullptr,
+                                     const void* up_in = nullptr);
 
 // The same on the tensor cores (bf16, segments of whole 64-row tiles); cudaErrorNotSupported otherwise.
 cudaError_t launch_ffn_backward_tc(const Dims& d, const void* x_perm, const int32_t* offsets, const void* W_gate,
                                    const void* W_up, const void* W_down, const void* h, const void* dy_perm,
                                    void* gate_buf, void* up_buf, void* dx_perm, float* dW_gate, float* dW_up,
-                                   float* dW_down, cudaStream_t st);
+                                   float* dW_down, cudaStream_t st, const void* gate_in = nullptr,
+                                   const void* up_in = nullptr);
 
 // C[r, :] = A[r, :] B[e]^T on the forward tensor-core kernel (A [M_cap, Kd], B [n_ffn, Nout, Kd], bf16)
 cudaError_t launch_grouped_gemm_tcgen05(const Dims& d, const void* A, const void* B, void* C, const int32_t* offsets,

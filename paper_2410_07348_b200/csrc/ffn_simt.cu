@@ -28,7 +28,8 @@ __device__ __forceinline__ void store1(__nv_bfloat16* p, float v) { *p = __float
 template <typename T, bool SWIGLU>
 __global__ void __launch_bounds__(256)
 ffn_simt_kernel(const T* __restrict__ A, const T* __restrict__ B0, const T* __restrict__ B1, T* __restrict__ C,
-                const int32_t* __restrict__ offsets, int n_ffn, int Nout, int Kd) {
+                const int32_t* __restrict__ offsets, int n_ffn, int Nout, int Kd, T* __restrict__ G,
+                T* __restrict__ U) {
   __shared__ float As[BK][BM + 4];
   __shared__ float Bs0[BK][BN + 4];
   __shared__ float Bs1[SWIGLU ? BK : 1][BN + 4];
@@ -110,6 +111,10 @@ ffn_simt_kernel(const T* __restrict__ A, const T* __restrict__ B0, const T* __re
       const int n = n0 + tx * 4 + j;
       if (n >= Nout) continue;
       float val = acc0[i][j];
+      if (SWIGLU && G != nullptr) {  // keep the pre-activations for the backward pass
+        store1(G + (size_t)r * Nout + n, acc0[i][j]);
+        store1(U + (size_t)r * Nout + n, acc1[i][j]);
+      }
       if (SWIGLU) val = (val / (1.f + expf(-val))) * acc1[i][j];
       store1(C + (size_t)r * Nout + n, val);
     }
@@ -118,26 +123,29 @@ ffn_simt_kernel(const T* __restrict__ A, const T* __restrict__ B0, const T* __re
 
 template <typename T>
 cudaError_t launch_t(const Dims& d, const void* x_perm, const int32_t* offsets, const void* W_gate, const void* W_up,
-                     const void* W_down, void* h, void* y_perm, cudaStream_t st) {
+                     const void* W_down, void* h, void* y_perm, cudaStream_t st, void* gate_out, void* up_out) {
   const unsigned mt = (unsigned)((d.M_cap + BM - 1) / BM + d.n_ffn);
   dim3 g1(mt, (unsigned)((d.F + BN - 1) / BN)), g2(mt, (unsigned)((d.D + BN - 1) / BN));
   ffn_simt_kernel<T, true><<<g1, 256, 0, st>>>(static_cast<const T*>(x_perm), static_cast<const T*>(W_gate),
                                                static_cast<const T*>(W_up), static_cast<T*>(h), offsets, d.n_ffn,
-                                               d.F, d.D);
+                                               d.F, d.D, static_cast<T*>(gate_out), static_cast<T*>(up_out));
   cudaError_t err = cudaGetLastError();
   if (err != cudaSuccess) return err;
   ffn_simt_kernel<T, false><<<g2, 256, 0, st>>>(static_cast<const T*>(h), static_cast<const T*>(W_down), nullptr,
-                                                static_cast<T*>(y_perm), offsets, d.n_ffn, d.D, d.F);
+                                                static_cast<T*>(y_perm), offsets, d.n_ffn, d.D, d.F, nullptr,
+                                                nullptr);
   return cudaGetLastError();
 }
 
 }  // namespace
 
 cudaError_t launch_ffn_simt(const Dims& d, const void* x_perm, const int32_t* offsets, const void* W_gate,
-                            const void* W_up, const void* W_down, void* h, void* y_perm, cudaStream_t st) {
+                            const void* W_up, const void* W_down, void* h, void* y_perm, cudaStream_t st,
+                            void* gate_out, void* up_out) {
   if (d.T == 0 || d.n_ffn == 0 || d.M_cap == 0) return cudaSuccess;
-  return d.dtype == MOEPP_BF16 ? launch_t<__nv_bfloat16>(d, x_perm, offsets, W_gate, W_up, W_down, h, y_perm, st)
-                               : launch_t<float>(d, x_perm, offsets, W_gate, W_up, W_down, h, y_perm, st);
+  return d.dtype == MOEPP_BF16
+             ? launch_t<__nv_bfloat16>(d, x_perm, offsets, W_gate, W_up, W_down, h, y_perm, st, gate_out, up_out)
+             : launch_t<float>(d, x_perm, offsets, W_gate, W_up, W_down, h, y_perm, st, gate_out, up_out);
 }
 
 }  // namespace moepp

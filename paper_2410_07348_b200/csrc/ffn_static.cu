@@ -85,8 +85,9 @@ extern "C" moepp_status moepp_grouped_ffn_static(const moepp_config* c, const vo
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   cudaError_t e;
   if (d.dtype == MOEPP_BF16 && !(d.flags & MOEPP_FLAG_SIMT_FFN)) {
-    e = ((d.flags & MOEPP_FLAG_FFN_SINGLE_CTA) ? launch_ffn_tcgen05 : launch_ffn_tcgen05_pair)(
-        d, x_perm, expert_offsets, W_gate, W_up, W_down, h, y_perm, st);
+    e = (d.flags & MOEPP_FLAG_FFN_SINGLE_CTA)
+            ? launch_ffn_tcgen05(d, x_perm, expert_offsets, W_gate, W_up, W_down, h, y_perm, st)
+            : launch_ffn_tcgen05_pair(d, x_perm, expert_offsets, W_gate, W_up, W_down, h, y_perm, st);
     if (e == cudaErrorNotSupported) return MOEPP_ERR_UNSUPPORTED;
   } else {
     e = launch_ffn_simt(d, x_perm, expert_offsets, W_gate, W_up, W_down, h, y_perm, st);

@@ -81,7 +81,8 @@ template <bool SWIGLU>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads2, 1)
 grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                          const __grid_constant__ CUtensorMap tmB1, __nv_bfloat16* __restrict__ C,
-                         const int32_t* __restrict__ offsets, int n_ffn, int Nout, int Kd, int32_t* err_word) {
+                         const int32_t* __restrict__ offsets, int n_ffn, int Nout, int Kd, int32_t* err_word,
+                         __nv_bfloat16* __restrict__ G, __nv_bfloat16* __restrict__ U) {
   constexpr int BN_OUT = SWIGLU ? 128 : 256;
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar_full[kStages2], bar_empty[kStages2], bar_tmem_full[2], bar_tmem_empty[2],
@@ -243,6 +244,23 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
           if (row_ok) {
             if (ti.n0 + c + 8 <= Nout) *reinterpret_cast<uint4*>(crow + c) = make_uint4(o[0], o[1], o[2], o[3]);
             if (ti.n0 + c + 16 <= Nout) *reinterpret_cast<uint4*>(crow + c + 8) = make_uint4(o[4], o[5], o[6], o[7]);
+            if (G != nullptr) {  // keep the pre-activations for the backward pass
+              uint32_t pg[8], pu[8];
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                pg[i] = pack_bf16(__uint_as_float(g[2 * i]), __uint_as_float(g[2 * i + 1]));
+                pu[i] = pack_bf16(__uint_as_float(u[2 * i]), __uint_as_float(u[2 * i + 1]));
+              }
+              const size_t at = (size_t)grow * Nout + ti.n0 + c;
+              if (ti.n0 + c + 8 <= Nout) {
+                *reinterpret_cast<uint4*>(G + at) = make_uint4(pg[0], pg[1], pg[2], pg[3]);
+                *reinterpret_cast<uint4*>(U + at) = make_uint4(pu[0], pu[1], pu[2], pu[3]);
+              }
+              if (ti.n0 + c + 16 <= Nout) {
+                *reinterpret_cast<uint4*>(G + at + 8) = make_uint4(pg[4], pg[5], pg[6], pg[7]);
+                *reinterpret_cast<uint4*>(U + at + 8) = make_uint4(pu[4], pu[5], pu[6], pu[7]);
+              }
+            }
           }
         }
       } else {
@@ -290,7 +308,8 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
 }  // namespace
 
 cudaError_t launch_ffn_tcgen05_pair(const Dims& d, const void* x_perm, const int32_t* offsets, const void* W_gate,
-                                    const void* W_up, const void* W_down, void* h, void* y_perm, cudaStream_t st) {
+                                    const void* W_up, const void* W_down, void* h, void* y_perm, cudaStream_t st,
+                                    void* gate_out, void* up_out) {
   if (d.T == 0 || d.n_ffn == 0 || d.M_cap == 0) return cudaSuccess;
   int dev = 0, sms = 0;
   cudaError_t err = cudaGetDevice(&dev);
@@ -340,11 +359,12 @@ cudaError_t launch_ffn_tcgen05_pair(const Dims& d, const void* x_perm, const int
   }
   const unsigned grid = (unsigned)(2 * pairs);
   k1<<<grid, kThreads2, kSmemBytes2, st>>>(mA1, mG, mU, static_cast<__nv_bfloat16*>(h), offsets, d.n_ffn, d.F, d.D,
-                                            err_word);
+                                            err_word, static_cast<__nv_bfloat16*>(gate_out),
+                                            static_cast<__nv_bfloat16*>(up_out));
   err = cudaGetLastError();
   if (err != cudaSuccess) return err;
   k2<<<grid, kThreads2, kSmemBytes2, st>>>(mA2, mD, mD, static_cast<__nv_bfloat16*>(y_perm), offsets, d.n_ffn, d.D,
-                                            d.F, err_word);
+                                            d.F, err_word, nullptr, nullptr);
   return cudaGetLastError();
 }
 

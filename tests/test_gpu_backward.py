@@ -110,6 +110,26 @@ def test_backward_random_shapes(oracle64, seed):
     check_backward(oracle64, lt, seed=seed, **over)
 
 
+@pytest.mark.parametrize("dtype,flags", [("f32", 0), ("bf16", 0), ("bf16", B.FLAG_SIMT_FFN)])
+def test_backward_with_kept_pre_activations(oracle64, dtype, flags):
+    """MOEPP_FLAG_SAVE_PREACT: the forward pass stores gate and up, the backward pass reads them instead of
+    recomputing; same oracle, same tolerance, and the forward output is unchanged by the flag."""
+    spec = W.LayerSpec(T=1500, D=200, F=328, n_ffn=4, n_zero=1, n_copy=1, n_const=1, top_k=2, dtype=dtype)
+    lt = W.make_layer(spec, seed=11, with_prev=True, w_std=0.05)
+    check_backward(oracle64, lt, row_align=64, flags=flags | B.FLAG_SAVE_PREACT)
+    wd = B.weights_from_tensors(lt)
+    x, prev = lt.x.cuda(), lt.prev.cuda()
+    ys = []
+    for fl in (flags, flags | B.FLAG_SAVE_PREACT):
+        cfg = B.config_from_spec(spec, row_align=64, flags=fl)
+        ws = torch.empty(B.moepp_workspace_bytes(cfg), dtype=torch.uint8, device="cuda")
+        y = torch.empty_like(x)
+        B.moepp_layer_forward(cfg, wd, x, prev, y, None, ws)
+        ys.append(y)
+    torch.cuda.synchronize()
+    assert torch.equal(ys[0], ys[1])
+
+
 def test_backward_no_tokens():
     spec = W.LayerSpec(T=0, D=64, F=96, n_ffn=2, n_zero=1, n_copy=1, n_const=1, top_k=2, dtype="f32")
     lt = W.make_layer(spec, seed=0, with_prev=True)
