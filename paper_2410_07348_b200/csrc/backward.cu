@@ -244,14 +244,15 @@ token_outer_kernel(const float* __restrict__ A, const TB* __restrict__ B, float*
     }
 }
 
-// out[i] = sum over z (in order) of part[z, i]
-__global__ void __launch_bounds__(256) sum_parts_kernel(const float* __restrict__ part, float* __restrict__ out,
-                                                        long long n, int Z) {
+// sum over z (in order) of part[z, i], written to out_a[i] for i < n_a and to out_b[i - n_a] after that
+__global__ void __launch_bounds__(256) sum_parts_kernel(const float* __restrict__ part, float* __restrict__ out_a,
+                                                        long long n_a, float* __restrict__ out_b, long long n, int Z) {
   const long long i = (long long)blockIdx.x * 256 + threadIdx.x;
   if (i >= n) return;
   float s = 0.f;
   for (int z = 0; z < Z; ++z) s += part[(size_t)z * n + i];
-  out[i] = s;
+  if (i < n_a) out_a[i] = s;
+  else out_b[i - n_a] = s;
 }
 
 // out[i] = sum over tokens of A[t, i]; one block per column, fixed order of the partial sums
@@ -269,54 +270,92 @@ __global__ void __launch_bounds__(256) column_sum_kernel(const float* __restrict
   if (threadIdx.x == 0) out[blockIdx.x] = s[0];
 }
 
-constexpr int kDxTokens = 8;  // tokens per warp in dx_assemble
+constexpr int kDxTokens = 4;   // tokens per warp in dx_assemble
+constexpr int kDxSlab = 256;   // columns per block
+constexpr int kDxGroups = 4;   // groups of 32 tokens a block serves one after the other
 
 // dx = cx dy + sum_r dGz[t, r] Wrow_r + sum over kept FFN picks of dXp[row_k, :],
 // Wrow_r = W_r[r, :] for r < N and the flattened W_c rows after that.
-// One warp owns kDxTokens tokens and walks the columns 256 at a time (8 per lane), so that every weight row it
-// reads is used for all its tokens.
+// A block owns 256 columns (blockIdx.y) of 128 tokens (blockIdx.x): the R x 256 slab of the stacked weights is
+// staged in shared memory once; the block then serves four groups of 32 tokens, each warp kDxTokens of them, a lane
+// holding columns 4 lane .. 4 lane + 3 and 128 + 4 lane .. of the slab (conflict-free 16-byte shared loads).
 template <typename XT>
-__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+__global__ void __launch_bounds__(kWarpsPerBlock * 32, 3)
 dx_assemble_kernel(Dims dm, int R, const XT* __restrict__ dy, const float* __restrict__ cx,
                    const float* __restrict__ dGz, const float* __restrict__ W_r, const float* __restrict__ W_c,
                    const XT* __restrict__ dXp, const int32_t* __restrict__ topk_idx,
                    const int32_t* __restrict__ row_of_slot, XT* __restrict__ dx) {
-  extern __shared__ float s_dx[];  // per warp: [R][kDxTokens] coefficients, then [kDxTokens] cx, then rows
+  extern __shared__ __align__(16) float s_dx[];  // [R][256] weights; per warp [R][kDxTokens] coefficients
   const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
   const int D = dm.D, N = dm.N, K = dm.K;
-  const int per_warp = R * kDxTokens + kDxTokens + kDxTokens * kMaxTopK;
-  float* s_c = s_dx + (size_t)wib * per_warp;
-  float* s_cx = s_c + R * kDxTokens;
-  int* s_rows = reinterpret_cast<int*>(s_cx + kDxTokens);
-  const long long t0 = ((long long)blockIdx.x * kWarpsPerBlock + wib) * kDxTokens;
-  if (t0 >= dm.T) return;
-  const int nt = (int)min((long long)kDxTokens, dm.T - t0);
-  for (int i = lane; i < R * kDxTokens; i += 32) {
-    const int r = i / kDxTokens, j = i % kDxTokens;
-    s_c[i] = j < nt ? dGz[(t0 + j) * R + r] : 0.f;
+  const int d0 = blockIdx.y * kDxSlab;
+  float* s_w = s_dx;
+  float* s_c = s_dx + (size_t)R * kDxSlab + (size_t)wib * R * kDxTokens;
+  for (int i = threadIdx.x; i < R * (kDxSlab / 4); i += kWarpsPerBlock * 32) {
+    const int r = i / (kDxSlab / 4), c4 = (i % (kDxSlab / 4)) * 4;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (d0 + c4 < D) {
+      const float* wrow = r < N ? W_r + (size_t)r * D : W_c + (size_t)(r - N) * D;
+      v = __ldg(reinterpret_cast<const float4*>(wrow + d0 + c4));
+    }
+    *reinterpret_cast<float4*>(s_w + (size_t)r * kDxSlab + c4) = v;
   }
-  for (int i = lane; i < kDxTokens * kMaxTopK; i += 32) {
-    const int j = i / kMaxTopK, k = i % kMaxTopK;
-    int row = -1;
-    if (j < nt && k < K && topk_idx[(t0 + j) * K + k] < dm.n_ffn) row = row_of_slot[(t0 + j) * K + k];  // -2: dropped
-    s_rows[i] = row;
-  }
-  if (lane < kDxTokens) s_cx[lane] = lane < nt ? cx[t0 + lane] : 0.f;
-  __syncwarp();
-  for (int d = lane * 8; d < D; d += 256) {
+  __syncthreads();
+  // the two 4-column groups of this lane
+  const int ca = d0 + 4 * lane, cb = d0 + 128 + 4 * lane;
+  const bool a_ok = ca < D, b_ok = cb < D;  // D is a multiple of 8, groups are 4-aligned
+  auto load4 = [&](const XT* p, float (&v)[4]) {
+    if (sizeof(XT) == 2) {
+      const uint2 u = *reinterpret_cast<const uint2*>(p);
+      v[0] = bf16_lo(u.x); v[1] = bf16_hi(u.x); v[2] = bf16_lo(u.y); v[3] = bf16_hi(u.y);
+    } else {
+      const float4 f = *reinterpret_cast<const float4*>(p);
+      v[0] = f.x; v[1] = f.y; v[2] = f.z; v[3] = f.w;
+    }
+  };
+  for (int grp = 0; grp < kDxGroups; ++grp) {
+    const long long t0 = (((long long)blockIdx.x * kDxGroups + grp) * kWarpsPerBlock + wib) * kDxTokens;
+    if (t0 >= dm.T) break;
+    const int nt = (int)min((long long)kDxTokens, dm.T - t0);
+    __syncwarp();
+    for (int i = lane; i < R * kDxTokens; i += 32) {
+      const int r = i / kDxTokens, j = i % kDxTokens;
+      s_c[i] = j < nt ? dGz[(t0 + j) * R + r] : 0.f;
+    }
+    __syncwarp();
+    // accumulators start from cx dy + the grouped rows of the kept FFN picks
     float acc[kDxTokens][8];
 #pragma unroll
-    for (int j = 0; j < kDxTokens; ++j)
+    for (int j = 0; j < kDxTokens; ++j) {
 #pragma unroll
       for (int i = 0; i < 8; ++i) acc[j][i] = 0.f;
+      if (j < nt) {
+        const float c = cx[t0 + j];
+        float va[4] = {0.f, 0.f, 0.f, 0.f}, vb[4] = {0.f, 0.f, 0.f, 0.f};
+        const XT* src = dy + (size_t)(t0 + j) * D;
+        if (a_ok) load4(src + ca, va);
+        if (b_ok) load4(src + cb, vb);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { acc[j][i] = c * va[i]; acc[j][4 + i] = c * vb[i]; }
+        for (int k = 0; k < K; ++k) {
+          if (topk_idx[(t0 + j) * K + k] >= dm.n_ffn) continue;
+          const int row = row_of_slot[(t0 + j) * K + k];  // -2: dropped
+          if (row < 0) continue;
+          src = dXp + (size_t)row * D;
+          if (a_ok) load4(src + ca, va);
+          if (b_ok) load4(src + cb, vb);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) { if (a_ok) acc[j][i] += va[i]; if (b_ok) acc[j][4 + i] += vb[i]; }
+        }
+      }
+    }
+#pragma unroll 4
     for (int r = 0; r < R; ++r) {
-      const float* wrow = r < N ? W_r + (size_t)r * D + d : W_c + (size_t)(r - N) * D + d;
-      const float4 a = __ldg(reinterpret_cast<const float4*>(wrow));
-      const float4 b = __ldg(reinterpret_cast<const float4*>(wrow + 4));
+      const float4 a = *reinterpret_cast<const float4*>(s_w + (size_t)r * kDxSlab + 4 * lane);
+      const float4 b = *reinterpret_cast<const float4*>(s_w + (size_t)r * kDxSlab + 128 + 4 * lane);
       const float wv[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
       const float4 c0 = *reinterpret_cast<const float4*>(s_c + r * kDxTokens);
-      const float4 c1 = *reinterpret_cast<const float4*>(s_c + r * kDxTokens + 4);
-      const float cj[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+      const float cj[4] = {c0.x, c0.y, c0.z, c0.w};
 #pragma unroll
       for (int j = 0; j < kDxTokens; ++j)
 #pragma unroll
@@ -324,80 +363,80 @@ dx_assemble_kernel(Dims dm, int R, const XT* __restrict__ dy, const float* __res
     }
 #pragma unroll
     for (int j = 0; j < kDxTokens; ++j) {
-      if (j < nt) {
-        float tmp[8];
-        const float c = s_cx[j];
-        Vec8<XT>::load(dy + (size_t)(t0 + j) * D + d, tmp);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) acc[j][i] = fmaf(c, tmp[i], acc[j][i]);
-        for (int k = 0; k < K; ++k) {
-          const int row = s_rows[j * kMaxTopK + k];
-          if (row >= 0) {
-            Vec8<XT>::load(dXp + (size_t)row * D + d, tmp);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) acc[j][i] += tmp[i];
-          }
-        }
-        Vec8<XT>::store(dx + (size_t)(t0 + j) * D + d, acc[j]);
+      if (j >= nt) continue;
+      XT* dst = dx + (size_t)(t0 + j) * D;
+      if (sizeof(XT) == 2) {
+        if (a_ok) *reinterpret_cast<uint2*>(dst + ca) = make_uint2(pack_bf16(acc[j][0], acc[j][1]), pack_bf16(acc[j][2], acc[j][3]));
+        if (b_ok) *reinterpret_cast<uint2*>(dst + cb) = make_uint2(pack_bf16(acc[j][4], acc[j][5]), pack_bf16(acc[j][6], acc[j][7]));
+      } else {
+        if (a_ok) *reinterpret_cast<float4*>(dst + ca) = make_float4(acc[j][0], acc[j][1], acc[j][2], acc[j][3]);
+        if (b_ok) *reinterpret_cast<float4*>(dst + cb) = make_float4(acc[j][4], acc[j][5], acc[j][6], acc[j][7]);
       }
     }
   }
 }
 
-constexpr int kRt = 12;  // rows of the small factor per pass in token_outer_rows
+constexpr int kOuterThreads = 128;
 
 // part[z, m, n] = sum over the tokens t of chunk z of A[t, m] * B[t, n] for a SMALL M (a few dozen rows) and a wide,
-// 8-aligned Nout: each thread keeps kRt x 4 sums for 4 columns, the block covers 1024 columns, and the rows of A
-// are taken kRt at a time (the chunk of B is read again from cache for each group).
-template <typename TB>
-__global__ void __launch_bounds__(256)
+// 8-aligned Nout: each thread keeps RT x 4 sums for 4 columns, the block covers 512 columns, and the rows of A
+// are taken RT at a time (one pass when M <= RT; otherwise the chunk of B is read again from cache per group).
+template <typename TB, int RT>
+__global__ void __launch_bounds__(kOuterThreads)
 token_outer_rows_kernel(const float* __restrict__ A, const TB* __restrict__ B, float* __restrict__ part, int T, int M,
                         int Nout, long long a_rs, long long b_rs, int chunk) {
   constexpr int TS = 32;  // tokens staged per trip
-  __shared__ __align__(16) float s_a[TS][kRt];
-  const int z = blockIdx.y, n = (blockIdx.x * 256 + threadIdx.x) * 4;
+  __shared__ __align__(16) float s_a[TS][RT];
+  const int z = blockIdx.y, n = (blockIdx.x * kOuterThreads + threadIdx.x) * 4;
   const int t_begin = z * chunk, t_end = min(T, t_begin + chunk);
   const bool col_ok = n < Nout;  // Nout is a multiple of 4
-  for (int m0 = 0; m0 < M; m0 += kRt) {
-    float acc[kRt][4];
+  for (int m0 = 0; m0 < M; m0 += RT) {
+    float acc[RT][4];
 #pragma unroll
-    for (int r = 0; r < kRt; ++r) acc[r][0] = acc[r][1] = acc[r][2] = acc[r][3] = 0.f;
+    for (int r = 0; r < RT; ++r) acc[r][0] = acc[r][1] = acc[r][2] = acc[r][3] = 0.f;
     for (int ts = t_begin; ts < t_end; ts += TS) {
       __syncthreads();
-      for (int i = threadIdx.x; i < TS * kRt; i += 256) {
-        const int tt = i / kRt, r = i % kRt;
+      for (int i = threadIdx.x; i < TS * RT; i += kOuterThreads) {
+        const int tt = i / RT, r = i % RT;
         s_a[tt][r] = (ts + tt < t_end && m0 + r < M) ? A[(size_t)(ts + tt) * a_rs + m0 + r] : 0.f;
       }
       __syncthreads();
       if (col_ok) {
-#pragma unroll 4
-        for (int tt = 0; tt < TS; ++tt) {
-          float bv[4] = {0.f, 0.f, 0.f, 0.f};
-          if (ts + tt < t_end) {
-            const TB* bp = B + (size_t)(ts + tt) * b_rs + n;
-            if (sizeof(TB) == 2) {
-              const uint2 u = *reinterpret_cast<const uint2*>(bp);
-              bv[0] = bf16_lo(u.x); bv[1] = bf16_hi(u.x); bv[2] = bf16_lo(u.y); bv[3] = bf16_hi(u.y);
-            } else {
-              const float4 f = *reinterpret_cast<const float4*>(bp);
-              bv[0] = f.x; bv[1] = f.y; bv[2] = f.z; bv[3] = f.w;
+#pragma unroll
+        for (int t8 = 0; t8 < TS; t8 += 8) {
+          float bv[8][4];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {  // eight independent loads in flight
+            bv[j][0] = bv[j][1] = bv[j][2] = bv[j][3] = 0.f;
+            if (ts + t8 + j < t_end) {
+              const TB* bp = B + (size_t)(ts + t8 + j) * b_rs + n;
+              if (sizeof(TB) == 2) {
+                const uint2 u = *reinterpret_cast<const uint2*>(bp);
+                bv[j][0] = bf16_lo(u.x); bv[j][1] = bf16_hi(u.x); bv[j][2] = bf16_lo(u.y); bv[j][3] = bf16_hi(u.y);
+              } else {
+                const float4 f = *reinterpret_cast<const float4*>(bp);
+                bv[j][0] = f.x; bv[j][1] = f.y; bv[j][2] = f.z; bv[j][3] = f.w;
+              }
             }
           }
 #pragma unroll
-          for (int r4 = 0; r4 < kRt; r4 += 4) {
-            const float4 av = *reinterpret_cast<const float4*>(&s_a[tt][r4]);
-            const float ar[4] = {av.x, av.y, av.z, av.w};
+          for (int j = 0; j < 8; ++j) {
 #pragma unroll
-            for (int r = 0; r < 4; ++r)
+            for (int r4 = 0; r4 < RT; r4 += 4) {
+              const float4 av = *reinterpret_cast<const float4*>(&s_a[t8 + j][r4]);
+              const float ar[4] = {av.x, av.y, av.z, av.w};
 #pragma unroll
-              for (int i = 0; i < 4; ++i) acc[r4 + r][i] = fmaf(ar[r], bv[i], acc[r4 + r][i]);
+              for (int r = 0; r < 4; ++r)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[r4 + r][i] = fmaf(ar[r], bv[j][i], acc[r4 + r][i]);
+            }
           }
         }
       }
     }
     if (col_ok) {
 #pragma unroll
-      for (int r = 0; r < kRt; ++r)
+      for (int r = 0; r < RT; ++r)
         if (m0 + r < M)
           *reinterpret_cast<float4*>(part + ((size_t)z * M + m0 + r) * Nout + n) =
               make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
@@ -407,10 +446,10 @@ token_outer_rows_kernel(const float* __restrict__ A, const TB* __restrict__ B, f
 
 }  // namespace
 
-// The reductions over tokens run in at most 64 chunks of at least 512 tokens.
+// The reductions over tokens run in at most 128 chunks of at least 256 tokens.
 int backward_token_chunks(const Dims& d, int* chunk_tokens) {
-  int chunk = (d.T + 63) / 64;
-  if (chunk < 512) chunk = 512;
+  int chunk = (d.T + 127) / 128;
+  if (chunk < 256) chunk = 256;
   chunk = (chunk + kOk - 1) / kOk * kOk;
   if (chunk_tokens != nullptr) *chunk_tokens = chunk;
   return d.T > 0 ? (d.T + chunk - 1) / chunk : 1;
@@ -418,15 +457,18 @@ int backward_token_chunks(const Dims& d, int* chunk_tokens) {
 
 namespace {
 
+// out_a takes the first rows_a rows of the [M, Nout] product, out_b (if any) the rest
 template <typename TB>
 cudaError_t token_outer(const Dims& d, const float* A, long long a_rs, int M, const TB* B, long long b_rs, int Nout,
-                        float* part, float* out, cudaStream_t st) {
+                        float* part, float* out_a, int rows_a, float* out_b, cudaStream_t st) {
   if (M == 0 || Nout == 0) return cudaSuccess;
   int chunk;
   const int Z = backward_token_chunks(d, &chunk);
   if (Nout % 8 == 0 && Nout >= 256 && b_rs % 8 == 0) {
-    dim3 grid((unsigned)((Nout + 1023) / 1024), (unsigned)Z);
-    token_outer_rows_kernel<TB><<<grid, 256, 0, st>>>(A, B, part, d.T, M, Nout, a_rs, b_rs, chunk);
+    dim3 grid((unsigned)((Nout + 4 * kOuterThreads - 1) / (4 * kOuterThreads)), (unsigned)Z);
+    if (M <= 8) token_outer_rows_kernel<TB, 8><<<grid, kOuterThreads, 0, st>>>(A, B, part, d.T, M, Nout, a_rs, b_rs, chunk);
+    else if (M <= 16) token_outer_rows_kernel<TB, 16><<<grid, kOuterThreads, 0, st>>>(A, B, part, d.T, M, Nout, a_rs, b_rs, chunk);
+    else token_outer_rows_kernel<TB, 24><<<grid, kOuterThreads, 0, st>>>(A, B, part, d.T, M, Nout, a_rs, b_rs, chunk);
   } else {
     dim3 grid((unsigned)((M + kOm - 1) / kOm), (unsigned)((Nout + kOn - 1) / kOn), (unsigned)Z);
     token_outer_kernel<TB><<<grid, 256, 0, st>>>(A, B, part, d.T, M, Nout, a_rs, b_rs, chunk);
@@ -434,7 +476,7 @@ cudaError_t token_outer(const Dims& d, const float* A, long long a_rs, int M, co
   cudaError_t err = cudaGetLastError();
   if (err != cudaSuccess) return err;
   const long long n = (long long)M * Nout;
-  sum_parts_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(part, out, n, Z);
+  sum_parts_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(part, out_a, (long long)rows_a * Nout, out_b, n, Z);
   return cudaGetLastError();
 }
 
@@ -468,29 +510,30 @@ cudaError_t layer_backward_t(const Dims& d, const ForwardState& fs, const moepp_
                                    b.dXp, g.dW_gate, g.dW_up, g.dW_down, st, fs.gate, fs.up);
   if (err != cudaSuccess) return err;
 
-  // router and constant-expert weights: [dG | dz]^T x, rows 0..N-1 -> dW_r, the rest -> dW_c
-  // (both land in one [R, D] product; it is computed into `part` and split on the way out)
-  if ((err = token_outer<XT>(d, b.dGz, R, d.N, x, d.D, d.D, b.part, g.dW_r, st)) != cudaSuccess) return err;
+  // router and constant-expert weights in one product: [dG | dz]^T x, rows 0..N-1 -> dW_r, the rest -> dW_c
+  if ((err = token_outer<XT>(d, b.dGz, R, R, x, d.D, d.D, b.part, g.dW_r, d.N, g.dW_c, st)) != cudaSuccess) return err;
   if (d.n_const > 0) {
-    if ((err = token_outer<XT>(d, b.dGz + d.N, R, 2 * d.n_const, x, d.D, d.D, b.part, g.dW_c, st)) != cudaSuccess)
-      return err;
-    if ((err = token_outer<XT>(d, b.cvq, d.n_const, d.n_const, dy, d.D, d.D, b.part, g.dv, st)) != cudaSuccess)
+    if ((err = token_outer<XT>(d, b.cvq, d.n_const, d.n_const, dy, d.D, d.D, b.part, g.dv, d.n_const, nullptr, st)) !=
+        cudaSuccess)
       return err;
   }
   if (w.W_g != nullptr && g.dW_g != nullptr) {
-    if ((err = token_outer<float>(d, b.dGz, R, d.N, prev, d.N, d.N, b.part, g.dW_g, st)) != cudaSuccess) return err;
+    if ((err = token_outer<float>(d, b.dGz, R, d.N, prev, d.N, d.N, b.part, g.dW_g, d.N, nullptr, st)) != cudaSuccess)
+      return err;
   }
   if (g.dbias != nullptr) {
     column_sum_kernel<<<(unsigned)d.N, 256, 0, st>>>(b.dGz, g.dbias, d.T, R);
     if ((err = cudaGetLastError()) != cudaSuccess) return err;
   }
-  const unsigned dx_blocks = (unsigned)((d.T + kWarpsPerBlock * kDxTokens - 1) / (kWarpsPerBlock * kDxTokens));
-  const size_t dx_smem = sizeof(float) * kWarpsPerBlock * ((size_t)R * kDxTokens + kDxTokens + kDxTokens * kMaxTopK);
+  const int dx_tokens = kWarpsPerBlock * kDxTokens * kDxGroups;
+  const dim3 dx_grid((unsigned)((d.T + dx_tokens - 1) / dx_tokens),
+                     (unsigned)((d.D + kDxSlab - 1) / kDxSlab));
+  const size_t dx_smem = sizeof(float) * ((size_t)R * kDxSlab + (size_t)kWarpsPerBlock * R * kDxTokens);
   if (dx_smem > 48 * 1024) {
     err = cudaFuncSetAttribute(dx_assemble_kernel<XT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dx_smem);
     if (err != cudaSuccess) return err;
   }
-  dx_assemble_kernel<XT><<<dx_blocks, kWarpsPerBlock * 32, dx_smem, st>>>(
+  dx_assemble_kernel<XT><<<dx_grid, kWarpsPerBlock * 32, dx_smem, st>>>(
       d, R, dy, b.cx, b.dGz, w.W_r, w.W_c, static_cast<const XT*>(b.dXp), fs.topk_idx, fs.row_of_slot,
       static_cast<XT*>(g.dx));
   return cudaGetLastError();

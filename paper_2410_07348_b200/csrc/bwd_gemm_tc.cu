@@ -254,34 +254,75 @@ bwd_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant_
         const int grow = ti.row0 + q * 32 + lane;
         const bool row_ok = grow < ti.row_end;
         const size_t at = (size_t)(row_ok ? grow : 0) * a.Nout + ti.n0;
-#pragma unroll 1
-        for (int c = 0; c < BN; c += 16) {
-          uint32_t r[16];
-          tmem_ld16(t_row + c, r);
-          tmem_ld_wait();
-          tmem_ld_pin(r);
+        if (MODE == DH) {
+          // gate / up of the next 16 columns are fetched while the current 16 are worked on
+          uint4 gq[2], uq[2], gn[2], un[2];
+          auto fetch = [&](int c, uint4 (&g)[2], uint4 (&u)[2]) {
 #pragma unroll
-          for (int half = 0; half < 2; ++half) {
-            if (!row_ok || ti.n0 + c + 8 * half + 8 > a.Nout) continue;
-            float f[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(r[8 * half + i]);
-            if (MODE == DH) {
-              __nv_bfloat16* gp = a.gate + at + c + 8 * half;
-              __nv_bfloat16* up = a.up + at + c + 8 * half;
-              float g[8], u[8], dg[8], du[8];
-              Vec8<__nv_bfloat16>::load(a.gate_in + at + c + 8 * half, g);
-              Vec8<__nv_bfloat16>::load(a.up_in + at + c + 8 * half, u);
-#pragma unroll
-              for (int i = 0; i < 8; ++i) {
-                const float s = 1.f / (1.f + __expf(-g[i]));
-                dg[i] = f[i] * u[i] * (s + g[i] * s * (1.f - s));
-                du[i] = f[i] * g[i] * s;
+            for (int half = 0; half < 2; ++half) {
+              g[half] = make_uint4(0u, 0u, 0u, 0u);
+              u[half] = make_uint4(0u, 0u, 0u, 0u);
+              if (row_ok && ti.n0 + c + 8 * half + 8 <= a.Nout) {
+                g[half] = *reinterpret_cast<const uint4*>(a.gate_in + at + c + 8 * half);
+                u[half] = *reinterpret_cast<const uint4*>(a.up_in + at + c + 8 * half);
               }
-              Vec8<__nv_bfloat16>::store(gp, dg);
-              Vec8<__nv_bfloat16>::store(up, du);
-            } else {
-              Vec8<__nv_bfloat16>::store(static_cast<__nv_bfloat16*>(a.C) + at + c + 8 * half, f);
+            }
+          };
+          fetch(0, gq, uq);
+#pragma unroll 1
+          for (int c = 0; c < BN; c += 16) {
+            if (c + 16 < BN) fetch(c + 16, gn, un);
+            uint32_t r[16];
+            tmem_ld16(t_row + c, r);
+            tmem_ld_wait();
+            tmem_ld_pin(r);
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+              if (!row_ok || ti.n0 + c + 8 * half + 8 > a.Nout) continue;
+              const uint32_t gw[4] = {gq[half].x, gq[half].y, gq[half].z, gq[half].w};
+              const uint32_t uw[4] = {uq[half].x, uq[half].y, uq[half].z, uq[half].w};
+              uint32_t og[4], ou[4];
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                float dg2[2], du2[2];
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                  const float g = j ? bf16_hi(gw[i]) : bf16_lo(gw[i]);
+                  const float u = j ? bf16_hi(uw[i]) : bf16_lo(uw[i]);
+                  const float dh = __uint_as_float(r[8 * half + 2 * i + j]);
+                  const float sg = __fdividef(1.f, 1.f + __expf(-g));
+                  dg2[j] = dh * u * (sg + g * sg * (1.f - sg));
+                  du2[j] = dh * g * sg;
+                }
+                og[i] = pack_bf16(dg2[0], dg2[1]);
+                ou[i] = pack_bf16(du2[0], du2[1]);
+              }
+              *reinterpret_cast<uint4*>(a.gate + at + c + 8 * half) = make_uint4(og[0], og[1], og[2], og[3]);
+              *reinterpret_cast<uint4*>(a.up + at + c + 8 * half) = make_uint4(ou[0], ou[1], ou[2], ou[3]);
+            }
+            gq[0] = gn[0]; gq[1] = gn[1]; uq[0] = un[0]; uq[1] = un[1];
+          }
+        } else {
+#pragma unroll 1
+          for (int c = 0; c < BN; c += 32) {
+            uint32_t r0[16], r1[16];
+            tmem_ld16(t_row + c, r0);
+            tmem_ld16(t_row + c + 16, r1);
+            tmem_ld_wait();
+            tmem_ld_pin(r0);
+            tmem_ld_pin(r1);
+            uint32_t o[16];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              o[i] = pack_bf16(__uint_as_float(r0[2 * i]), __uint_as_float(r0[2 * i + 1]));
+              o[8 + i] = pack_bf16(__uint_as_float(r1[2 * i]), __uint_as_float(r1[2 * i + 1]));
+            }
+            if (row_ok) {
+              __nv_bfloat16* crow = static_cast<__nv_bfloat16*>(a.C) + at + c;
+#pragma unroll
+              for (int v = 0; v < 4; ++v)
+                if (ti.n0 + c + 8 * v + 8 <= a.Nout)
+                  *reinterpret_cast<uint4*>(crow + 8 * v) = make_uint4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
             }
           }
         }

@@ -130,6 +130,23 @@ def test_backward_with_kept_pre_activations(oracle64, dtype, flags):
     assert torch.equal(ys[0], ys[1])
 
 
+def test_backward_experts_without_rows_on_tensor_cores(oracle64):
+    """Fewer slots than experts: the weight-gradient tiles of an expert nobody picked have an empty k range and must
+    come out as exact zeros (bf16, 64-row segments, so the tensor-core kernels run)."""
+    spec = W.LayerSpec(T=5, D=128, F=256, n_ffn=12, n_zero=1, n_copy=1, n_const=1, top_k=2, dtype="bf16")
+    lt = W.make_layer(spec, seed=2, with_prev=True, w_std=0.05)
+    check_backward(oracle64, lt, row_align=64)
+    cfg = B.config_from_spec(spec, row_align=64)
+    wd = B.weights_from_tensors(lt)
+    dy = torch.ones(spec.T, spec.D, dtype=torch.bfloat16, device="cuda")
+    got, idx = gpu_backward(cfg, wd, lt.x.cuda(), lt.prev.cuda(), dy, None)
+    unused = [e for e in range(spec.n_ffn) if not (idx == e).any()]
+    assert unused
+    for e in unused:
+        for name in ("dW_gate", "dW_up", "dW_down"):
+            assert not np.any(got[name][e]), (name, e)
+
+
 def test_backward_no_tokens():
     spec = W.LayerSpec(T=0, D=64, F=96, n_ffn=2, n_zero=1, n_copy=1, n_const=1, top_k=2, dtype="f32")
     lt = W.make_layer(spec, seed=0, with_prev=True)
