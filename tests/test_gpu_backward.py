@@ -147,6 +147,61 @@ def test_backward_experts_without_rows_on_tensor_cores(oracle64):
             assert not np.any(got[name][e]), (name, e)
 
 
+def test_backward_through_two_chained_layers(oracle64):
+    """Two layers joined by the residual stream and the gating residual (Eq. 6): layer 2's dx is layer 1's dy and
+    layer 2's dprev is the dlogits layer 1 receives.  GPU chain against the oracle's chain, float32."""
+    spec = W.LayerSpec(T=300, D=96, F=160, n_ffn=4, n_zero=1, n_copy=1, n_const=2, top_k=2, dtype="f32")
+    l1 = W.make_layer(spec, seed=21, with_prev=True, w_std=0.05)
+    l2 = W.make_layer(spec, seed=22, with_prev=True, w_std=0.05)
+    cfg = B.config_from_spec(spec, add_residual=1)
+    w1, w2 = B.weights_from_tensors(l1), B.weights_from_tensors(l2)
+    dev = "cuda"
+    x, prev = l1.x.cuda(), l1.prev.cuda()
+    T, N, D = spec.T, spec.N, spec.D
+    new = lambda *shape: torch.empty(*shape, device=dev)
+    ws1 = torch.empty(B.moepp_workspace_bytes(cfg), dtype=torch.uint8, device=dev)
+    ws2 = torch.empty_like(ws1)
+    bws = torch.empty(B.moepp_backward_workspace_bytes(cfg), dtype=torch.uint8, device=dev)
+    y1, g1, y2, g2 = new(T, D), new(T, N), new(T, D), new(T, N)
+    B.moepp_layer_forward(cfg, w1, x, prev, y1, g1, ws1)
+    B.moepp_layer_forward(cfg, w2, y1, g1, y2, g2, ws2)
+    gen = torch.Generator().manual_seed(5)
+    R, Q = torch.randn(T, D, generator=gen), 0.1 * torch.randn(T, N, generator=gen)
+
+    def grads():
+        return dict(dx=new(T, D), dprev=new(T, N), dW_r=new(N, D), dW_g=new(N, N), dbias=new(N),
+                    dW_c=new(spec.n_const, 2, D), dv=new(spec.n_const, D), dW_gate=new(spec.n_ffn, spec.F, D),
+                    dW_up=new(spec.n_ffn, spec.F, D), dW_down=new(spec.n_ffn, D, spec.F))
+
+    ga, gb = grads(), grads()
+    B.moepp_layer_backward(cfg, w2, y1, g1, g2, R.cuda(), Q.cuda(), ws2, gb, bws)
+    B.moepp_layer_backward(cfg, w1, x, prev, g1, gb["dx"], gb["dprev"], ws1, ga, bws)
+    idx = []
+    for (w, xin, pin) in ((w1, x, prev), (w2, y1, g1)):
+        i_ = torch.empty(T, spec.top_k, dtype=torch.int32, device=dev)
+        B.moepp_route(cfg, xin, w["W_r"], w["W_g"], pin, w["router_bias"], None, new(T, N), i_, new(T, spec.top_k),
+                      torch.empty(N, dtype=torch.int32, device=dev),
+                      torch.empty(spec.n_ffn + 1, dtype=torch.int32, device=dev), None)
+        idx.append(i_.cpu().numpy())
+    torch.cuda.synchronize()
+
+    # the oracle's own chain from the same x: forward both layers, backward both layers
+    s = shape_of(spec, add_residual=1)
+    o1, o2 = oracle_inputs(l1), oracle_inputs(l2)
+    f1 = oracle64.layer_forward(s, o1["x"], o1["W_r"], o1["W_g"], o1["prev"], o1["bias"], o1["W_c"], o1["v"], o1["W_gate"],
+                                o1["W_up"], o1["W_down"], forced_idx=idx[0])
+    b2 = oracle64.layer_backward(s, f1["y"], o2["W_r"], idx[1], f32(R), o2["W_g"], f1["logits"], o2["bias"], o2["W_c"],
+                                 o2["v"], o2["W_gate"], o2["W_up"], o2["W_down"], dlogits=f32(Q))
+    b1 = oracle64.layer_backward(s, o1["x"], o1["W_r"], idx[0], b2["dx"], o1["W_g"], o1["prev"], o1["bias"], o1["W_c"],
+                                 o1["v"], o1["W_gate"], o1["W_up"], o1["W_down"], dlogits=b2["dprev"])
+    for got, ref in ((gb, b2), (ga, b1)):
+        for name in GRADS:
+            r = ref[name]
+            scale = max(float(np.abs(r).max()), 1e-6)
+            err = float(np.abs(got[name].cpu().numpy().astype(np.float64) - r).max()) / scale
+            assert err <= 5e-4, (name, err)
+
+
 def test_backward_no_tokens():
     spec = W.LayerSpec(T=0, D=64, F=96, n_ffn=2, n_zero=1, n_copy=1, n_const=1, top_k=2, dtype="f32")
     lt = W.make_layer(spec, seed=0, with_prev=True)
