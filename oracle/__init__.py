@@ -153,6 +153,14 @@ class Oracle:
         self._call("balance_stats", self._cfg(s), _ptr(G), _ptr(idx), _ptr(f), _ptr(P), _ptr(loss))
         return f, P, float(loss[0])
 
+    def balance_backward(self, s, G, f, scale=1.0, into=None):
+        """d(scale * L_b)/dG of Eq. 7 with f held fixed; added to `into` (float32 [T, N]) if given."""
+        G, f = _f32(G), _f32(f)
+        dG = np.zeros((s.T, s.N), np.float32) if into is None else np.ascontiguousarray(into, np.float32).copy()
+        self._call("balance_backward", self._cfg(s), _ptr(G), _ptr(f), ctypes.c_float(scale),
+                   ctypes.c_int(0 if into is None else 1), _ptr(dG))
+        return dG
+
     def permute_rows(self, s, x, slot_of_row):
         x, slot_of_row = _f32(x), _i32(slot_of_row)
         out = np.empty((len(slot_of_row), s.D), np.float32)

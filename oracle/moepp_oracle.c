@@ -446,6 +446,34 @@ int FN(balance_stats)(const oracle_config* c, const float* G, const int32_t* idx
   return 0;
 }
 
+/* ---- Eq. 7 differentiated with respect to the router logits ----------------------------------------
+ * L_b = sum_i eta_i f_i P_i, P_i = (1/T) sum_t softmax(G_t)_i.  f_i counts selections and is piecewise
+ * constant in G, so only P_i carries a gradient:
+ *   d(scale L_b)/dG[t,j] = (scale/T) P_tj (c_j - sum_i c_i P_ti),  c_i = eta_i f_i.
+ * accumulate != 0 adds to dG instead of overwriting it. */
+int FN(balance_backward)(const oracle_config* c, const float* G, const float* f, float scale, int accumulate,
+                         float* dG) {
+  if (bad_config(c) || !G || !f || !dG) return 1;
+  const int N = n_experts(c);
+  if (N > 256) return 1;
+  const real tau = c->tau > 0.0f ? (real)c->tau : (real)1;
+  real ci[256];
+  for (int i = 0; i < N; ++i) ci[i] = (i < c->n_ffn ? (real)1 : tau) * (real)f[i];
+  for (int t = 0; t < c->T; ++t) {
+    real g[256], P[256];
+    for (int i = 0; i < N; ++i) g[i] = (real)G[(int64_t)t * N + i];
+    softmax_all(g, N, P);
+    real dot = 0;
+    for (int i = 0; i < N; ++i) dot += ci[i] * P[i];
+    for (int j = 0; j < N; ++j) {
+      const real v = (real)scale / (real)c->T * P[j] * (ci[j] - dot);
+      float* out = dG + (int64_t)t * N + j;
+      *out = accumulate ? (float)((real)*out + v) : (float)v;
+    }
+  }
+  return 0;
+}
+
 /* ==== backward pass: chain rule through Eq. 1-6, token by token ===================================== */
 
 /* gradient accumulators for the weights, in `real`, rounded to float once at the end */

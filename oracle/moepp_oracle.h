@@ -94,6 +94,8 @@ int oracle_num_threads(void);
      loss = sum_i eta_i f[i] P[i] with eta = 1 (FFN) or tau (zero-computation). */                           \
   int P##balance_stats(const oracle_config* c, const float* G, const int32_t* idx, float* f, float* Pm,     \
                        float* loss);                                                                        \
+  int P##balance_backward(const oracle_config* c, const float* G, const float* f, float scale,             \
+                          int accumulate, float* dG);                                                       \
   /* Whole layer by the definition, token by token, without any grouping.                          \
      tokens==NULL: all T tokens, y is [T,D]; else y is [n_tokens,D] for the listed tokens.         \
      forced_idx (may be NULL) replaces the top-K choice; the weights still come from the           \

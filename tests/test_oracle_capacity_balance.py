@@ -165,3 +165,57 @@ def test_balance_stats_against_torch(oracle64, oracle32):
     assert abs((L1 - L) - float((0.25 * ft[8:] * Pt[8:]).sum())) < 1e-6
     f32_, P32, L32 = oracle32.balance_stats(s, G, idx)
     assert abs(L32 - L) < 1e-5
+
+
+# ------------------------------------------------------------------------------------------------
+# Eq. 7 differentiated with respect to the logits (f held fixed)
+# ------------------------------------------------------------------------------------------------
+def _balance_problem(T=9, n_ffn=3, n_zero=1, n_copy=1, n_const=1, K=2, tau=0.6):
+    s = LayerShape(T=T, D=8, F=8, n_ffn=n_ffn, n_zero=n_zero, n_copy=n_copy, n_const=n_const, top_k=K, tau=tau)
+    G = _rand(T, s.N)
+    idx = np.stack([rng.permutation(s.N)[:K] for _ in range(T)]).astype(np.int32)
+    return s, G, idx
+
+
+def test_balance_backward_matches_finite_differences(oracle64):
+    s, G, idx = _balance_problem()
+    f, _, _ = oracle64.balance_stats(s, G, idx)
+    dG = oracle64.balance_backward(s, G, f, scale=0.7)
+    eps = 1e-2
+    for t, j in [(0, 0), (3, 2), (8, 5), (4, 4), (7, 1)]:
+        keep = G[t, j]
+        G[t, j] = keep + eps
+        hi = oracle64.balance_stats(s, G, idx)[2]
+        G[t, j] = keep - eps
+        lo = oracle64.balance_stats(s, G, idx)[2]
+        G[t, j] = keep
+        step = float(np.float32(keep + eps)) - float(np.float32(keep - eps))
+        assert abs(0.7 * (hi - lo) / step - dG[t, j]) < 2e-5, (t, j)
+
+
+def test_balance_backward_matches_torch_autograd(oracle64):
+    s, G, idx = _balance_problem(T=17, n_ffn=5, n_const=2, tau=0.25)
+    f, _, _ = oracle64.balance_stats(s, G, idx)
+    g = torch.tensor(G, dtype=torch.float64, requires_grad=True)
+    eta = torch.tensor([1.0] * s.n_ffn + [0.25] * (s.N - s.n_ffn), dtype=torch.float64)
+    loss = (eta * torch.tensor(f, dtype=torch.float64) * torch.softmax(g, dim=1).mean(dim=0)).sum()
+    loss.backward()
+    dG = oracle64.balance_backward(s, G, f, scale=1.0)
+    assert np.abs(dG - g.grad.numpy()).max() < 1e-8
+    # every row sums to zero: a constant added to a token's logits changes nothing
+    assert np.abs(dG.sum(axis=1)).max() < 1e-8
+    # accumulation adds to what is there
+    base = _rand(s.T, s.N)
+    acc = oracle64.balance_backward(s, G, f, scale=2.0, into=base)
+    assert np.abs(acc - (base + 2.0 * dG)).max() < 1e-6
+
+
+def test_balance_backward_closed_form_for_equal_logits(oracle64):
+    # equal logits: P = 1/N everywhere, so dG[t, j] = scale / (T N) * (c_j - mean(c)), c_i = eta_i f_i
+    s, _, idx = _balance_problem(T=6, tau=0.5)
+    G = np.full((s.T, s.N), 0.3, np.float32)
+    f, _, _ = oracle64.balance_stats(s, G, idx)
+    c = np.array([1.0] * s.n_ffn + [0.5] * (s.N - s.n_ffn)) * f.astype(np.float64)
+    want = 3.0 / (s.T * s.N) * (c - c.mean())
+    dG = oracle64.balance_backward(s, G, f, scale=3.0)
+    assert np.abs(dG - want[None, :]).max() < 1e-8
