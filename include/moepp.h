@@ -192,6 +192,17 @@ moepp_status moepp_balance_stats(const moepp_config* cfg, const float* logits, c
                                  float* P, float* loss, void* stream);
 
 /*
+ * Gradient of scale * L_b (Eq. 7; the paper adds beta * L_b to the training loss, Sec. 3.4) with respect to
+ * the router logits.  f_i only counts selections, so it is held fixed and the gradient flows through P_i:
+ *   dlogits[t, j] (+)= (scale / T) P_tj (c_j - sum_i c_i P_ti),  P_t = softmax(logits[t, :]),  c_i = eta_i f_i.
+ *   logits [T, N] float (device), f [N] float (device; what moepp_balance_stats wrote)
+ *   dlogits [T, N] float (device): overwritten, or added to when accumulate != 0 -- e.g. on top of the dprev
+ *   the next layer's moepp_layer_backward produced, before it is passed on as dlogits_next.
+ */
+moepp_status moepp_balance_backward(const moepp_config* cfg, const float* logits, const float* f, float scale,
+                                    int32_t accumulate, float* dlogits, void* stream);
+
+/*
  * A stack of n_layers layers that share one configuration (the gating residual of Eq. 6 carries the
  * logits from layer to layer): layer j reads x^j and the logits of layer j-1 and produces
  * x^{j+1} = (x^j if add_residual) + Eq. 1 and its own logits.  layers[j] holds layer j's weights; a layer

@@ -26,7 +26,7 @@ EXPORTS = ("moepp_status_string", "moepp_workspace_bytes", "moepp_workspace_byte
            "moepp_layer_forward_host", "moepp_device_error", "moepp_grouped_ffn_static",
            "moepp_stack_workspace_bytes", "moepp_stack_forward", "moepp_stack_workspace_bytes_host",
            "moepp_stack_forward_host", "moepp_balance_stats", "moepp_backward_workspace_bytes",
-           "moepp_layer_backward")
+           "moepp_layer_backward", "moepp_balance_backward")
 STATIC_SCRATCH_BYTES = 32 << 20
 
 
@@ -195,13 +195,20 @@ def moepp_layer_backward(cfg, weights: dict, x, prev_logits, logits, dy, dlogits
     nbytes = lambda t: ctypes.c_size_t(t.numel() * t.element_size())
     _check(lib().moepp_layer_backward(ctypes.byref(c), ctypes.byref(w), _p(x), _p(prev_logits), _p(logits), _p(dy),
                                       _p(dlogits_next), _p(fwd_workspace), nbytes(fwd_workspace), ctypes.byref(g),
-                                      _p(bwd_workspace), nbytes(bwd_workspace), _stream()), "moepp_layer_backward")
+                                      _p(bwd_workspace), nbytes(bwd_workspace), _stream()), "moepp_layer_backward", "moepp_balance_backward")
 
 
 def moepp_balance_stats(cfg, logits, expert_counts, f, P, loss):
     c = cfg.c()
     _check(lib().moepp_balance_stats(ctypes.byref(c), _p(logits), _p(expert_counts), _p(f), _p(P), _p(loss),
                                      _stream()), "moepp_balance_stats")
+
+
+def moepp_balance_backward(cfg, logits, f, scale, dlogits, accumulate=False):
+    c = cfg.c()
+    _check(lib().moepp_balance_backward(ctypes.byref(c), _p(logits), _p(f), ctypes.c_float(scale),
+                                        ctypes.c_int32(1 if accumulate else 0), _p(dlogits), _stream()),
+           "moepp_balance_backward")
 
 
 def _weights_array(weights_list):

@@ -545,6 +545,17 @@ moepp_status moepp_balance_stats(const moepp_config* cfg, const float* logits, c
   return from_cuda(launch_balance_stats(d, logits, expert_counts, f, P, loss, static_cast<cudaStream_t>(stream)));
 }
 
+moepp_status moepp_balance_backward(const moepp_config* cfg, const float* logits, const float* f, float scale,
+                                    int32_t accumulate, float* dlogits, void* stream) {
+  Dims d;
+  const moepp_status s = make_dims(cfg, &d);
+  if (s != MOEPP_OK) return s;
+  if (f == nullptr) return MOEPP_ERR_INVALID_ARG;
+  if (d.T > 0 && (logits == nullptr || dlogits == nullptr)) return MOEPP_ERR_INVALID_ARG;
+  return from_cuda(launch_balance_backward(d, logits, f, scale, accumulate != 0, dlogits,
+                                           static_cast<cudaStream_t>(stream)));
+}
+
 // Device scratch of the backward pass, carved like the forward workspace.
 struct BwdCarve {
   size_t dYp, gate, up, dXp, dw, dGz, cx, cvq, part, total;

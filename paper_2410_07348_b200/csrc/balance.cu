@@ -65,7 +65,49 @@ balance_stats_kernel(Dims dm, const float* __restrict__ logits, const int32_t* _
   }
 }
 
+// Eq. 7 differentiated with respect to the logits, f held fixed (it only counts selections):
+//   d(scale L_b)/dG[t, j] = (scale / T) P_tj (c_j - sum_i c_i P_ti),  c_i = eta_i f_i.
+// One warp per token, lane l holds experts l and l + 32; written to dG or added to it.
+__global__ void __launch_bounds__(256)
+balance_bwd_kernel(Dims dm, const float* __restrict__ logits, const float* __restrict__ f, float scale,
+                   int accumulate, float* __restrict__ dG) {
+  const int lane = threadIdx.x & 31, N = dm.N;
+  const long long t = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (t >= dm.T) return;
+  const int i0 = lane, i1 = lane + 32;
+  const float g0 = i0 < N ? logits[t * N + i0] : -INFINITY, g1 = i1 < N ? logits[t * N + i1] : -INFINITY;
+  float m = fmaxf(g0, g1);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  const float e0 = i0 < N ? expf(g0 - m) : 0.f, e1 = i1 < N ? expf(g1 - m) : 0.f;
+  float z = e0 + e1;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
+  const float P0 = e0 / z, P1 = e1 / z;
+  const float c0 = i0 < N ? (i0 < dm.n_ffn ? 1.f : dm.tau) * f[i0] : 0.f;
+  const float c1 = i1 < N ? (i1 < dm.n_ffn ? 1.f : dm.tau) * f[i1] : 0.f;
+  float dot = c0 * P0 + c1 * P1;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+  const float k = scale / (float)dm.T;
+  if (i0 < N) {
+    const float v = k * P0 * (c0 - dot);
+    dG[t * N + i0] = accumulate ? dG[t * N + i0] + v : v;
+  }
+  if (i1 < N) {
+    const float v = k * P1 * (c1 - dot);
+    dG[t * N + i1] = accumulate ? dG[t * N + i1] + v : v;
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_balance_backward(const Dims& d, const float* logits, const float* f, float scale, int accumulate,
+                                    float* dlogits, cudaStream_t st) {
+  if (d.T == 0) return cudaSuccess;
+  balance_bwd_kernel<<<(unsigned)((d.T + 7) / 8), 256, 0, st>>>(d, logits, f, scale, accumulate, dlogits);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_balance_stats(const Dims& d, const float* logits, const int32_t* counts, float* f, float* P,
                                  float* loss, cudaStream_t st) {

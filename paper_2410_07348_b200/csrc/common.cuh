@@ -63,6 +63,9 @@ cudaError_t launch_ffn_tcgen05_pair(const Dims& d, const void* x_perm, const int
 cudaError_t launch_balance_stats(const Dims& d, const float* logits, const int32_t* counts, float* f, float* P,
                                  float* loss, cudaStream_t st);
 
+cudaError_t launch_balance_backward(const Dims& d, const float* logits, const float* f, float scale, int accumulate,
+                                    float* dlogits, cudaStream_t st);
+
 cudaError_t launch_combine(const Dims& d, const void* x, const void* y_perm, const int32_t* topk_idx,
                            const float* topk_w, const int32_t* row_of_slot, const float* alpha, const float* W_c,
                            const float* v, void* y, cudaStream_t st);

@@ -408,3 +408,24 @@ def test_balance_stats(oracle64):
         B.moepp_balance_stats(cfg, lg, cnt, f, P2, loss2)
         torch.cuda.synchronize()
         assert torch.equal(P, P2) and torch.equal(loss, loss2)
+
+
+def test_balance_backward(oracle64):
+    """Gradient of the Eq. 7 loss with respect to the logits (f held fixed): overwrite and accumulate forms."""
+    for spec, tau in ((W.CONFIGS["cfg1_tiny_f32"], 0.75), (W.LayerSpec(T=3001, D=64, F=64, n_ffn=40, n_const=8), 0.1)):
+        cfg = B.config_from_spec(spec, tau=tau)
+        s = shape_of(spec, tau=tau)
+        T, N = spec.T, spec.N
+        gen = torch.Generator().manual_seed(3)
+        lg = 2.0 * torch.randn(T, N, generator=gen)
+        f = torch.rand(N, generator=gen)
+        base = torch.randn(T, N, generator=gen)
+        out = torch.full((T, N), float("nan"), device="cuda")
+        B.moepp_balance_backward(cfg, lg.cuda(), f.cuda(), 0.01, out)
+        acc = base.cuda()
+        B.moepp_balance_backward(cfg, lg.cuda(), f.cuda(), 0.01, acc, accumulate=True)
+        torch.cuda.synchronize()
+        ref = oracle64.balance_backward(s, lg.numpy(), f.numpy(), scale=0.01)
+        scale = float(np.abs(ref).max())
+        assert max_abs(out.cpu().numpy(), ref) <= 1e-5 * scale + 1e-12
+        assert max_abs(acc.cpu().numpy(), base.numpy().astype(np.float64) + ref) <= 1e-6
