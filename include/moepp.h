@@ -275,6 +275,40 @@ moepp_status moepp_layer_backward(const moepp_config* cfg, const moepp_weights* 
                                   void* stream);
 
 /*
+ * The stack of moepp_stack_forward in a form that can be differentiated, and its backward pass: a training
+ * step's worth of the layer (the paper trains all layers jointly on the language-model loss plus beta times
+ * the sum of the layers' Eq. 7 losses, Sec. 3.4; it prints no backward formulas).
+ *
+ * moepp_stack_forward_train computes what moepp_stack_forward computes (same kernels, same bits) but gives every
+ * layer its own slot in `workspace` (moepp_stack_train_workspace_bytes: n_layers layer workspaces, outputs and
+ * logits), so that nothing a backward pass needs is overwritten.
+ *
+ * moepp_stack_backward walks the layers last to first with moepp_layer_backward's arithmetic: layer j's dx is
+ * layer j-1's dy, layer j's dprev is what reaches layer j-1's logits through Eq. 6.
+ *   x, prev_logits       the inputs the forward call had
+ *   dy [T, D]            dL/d(output of the last layer);  dlogits_last [T, N] or NULL: dL/d(its logits)
+ *   balance_scale        beta: if non-zero, beta * dL_b/dlogits (Eq. 7, moepp_balance_backward) of EVERY layer is
+ *                        added to that layer's logit gradient; balance_loss_out ([n_layers] float, device, may be
+ *                        NULL) then receives each layer's L_b
+ *   grads[n_layers]      one gradient set per layer, all weight gradients overwritten; dx and dprev are taken
+ *                        from grads[0] only (gradients with respect to x and prev_logits); the others' dx / dprev
+ *                        fields are ignored (the call keeps those intermediates in its own scratch)
+ *   bwd_workspace        moepp_stack_backward_workspace_bytes
+ * All pointers are device memory; nothing is allocated.  Flags as in moepp_layer_forward / moepp_layer_backward
+ * (MOEPP_FLAG_SAVE_PREACT must be the same in both calls).
+ */
+moepp_status moepp_stack_train_workspace_bytes(const moepp_config* cfg, int32_t n_layers, size_t* bytes);
+moepp_status moepp_stack_forward_train(const moepp_config* cfg, const moepp_weights* layers, int32_t n_layers,
+                                       const void* x, const float* prev_logits, void* y, float* logits_out,
+                                       void* workspace, size_t workspace_bytes, void* stream);
+moepp_status moepp_stack_backward_workspace_bytes(const moepp_config* cfg, int32_t n_layers, size_t* bytes);
+moepp_status moepp_stack_backward(const moepp_config* cfg, const moepp_weights* layers, int32_t n_layers, const void* x,
+                                  const float* prev_logits, const void* dy, const float* dlogits_last,
+                                  float balance_scale, float* balance_loss_out, const void* train_workspace,
+                                  size_t train_workspace_bytes, const moepp_grads* grads, void* bwd_workspace,
+                                  size_t bwd_workspace_bytes, void* stream);
+
+/*
  * moepp_grouped_ffn without a scratch argument.  (The paper has no counterpart to this call: it exists
  * for the way this library is embedded, not for the method.)
  *

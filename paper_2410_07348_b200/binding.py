@@ -26,7 +26,8 @@ EXPORTS = ("moepp_status_string", "moepp_workspace_bytes", "moepp_workspace_byte
            "moepp_layer_forward_host", "moepp_device_error", "moepp_grouped_ffn_static",
            "moepp_stack_workspace_bytes", "moepp_stack_forward", "moepp_stack_workspace_bytes_host",
            "moepp_stack_forward_host", "moepp_balance_stats", "moepp_backward_workspace_bytes",
-           "moepp_layer_backward", "moepp_balance_backward")
+           "moepp_layer_backward", "moepp_balance_backward", "moepp_stack_train_workspace_bytes",
+           "moepp_stack_forward_train", "moepp_stack_backward_workspace_bytes", "moepp_stack_backward")
 STATIC_SCRATCH_BYTES = 32 << 20
 
 
@@ -195,13 +196,58 @@ def moepp_layer_backward(cfg, weights: dict, x, prev_logits, logits, dy, dlogits
     nbytes = lambda t: ctypes.c_size_t(t.numel() * t.element_size())
     _check(lib().moepp_layer_backward(ctypes.byref(c), ctypes.byref(w), _p(x), _p(prev_logits), _p(logits), _p(dy),
                                       _p(dlogits_next), _p(fwd_workspace), nbytes(fwd_workspace), ctypes.byref(g),
-                                      _p(bwd_workspace), nbytes(bwd_workspace), _stream()), "moepp_layer_backward", "moepp_balance_backward")
+                                      _p(bwd_workspace), nbytes(bwd_workspace), _stream()), "moepp_layer_backward")
 
 
 def moepp_balance_stats(cfg, logits, expert_counts, f, P, loss):
     c = cfg.c()
     _check(lib().moepp_balance_stats(ctypes.byref(c), _p(logits), _p(expert_counts), _p(f), _p(P), _p(loss),
                                      _stream()), "moepp_balance_stats")
+
+
+def _grads(grads: dict) -> moepp_grads:
+    g = moepp_grads()
+    for name, _ in moepp_grads._fields_:
+        setattr(g, name, _p(grads.get(name)))
+    return g
+
+
+def moepp_stack_train_workspace_bytes(cfg: Config, n_layers: int) -> int:
+    n = ctypes.c_size_t(0)
+    c = cfg.c()
+    _check(lib().moepp_stack_train_workspace_bytes(ctypes.byref(c), ctypes.c_int32(n_layers), ctypes.byref(n)),
+           "moepp_stack_train_workspace_bytes")
+    return int(n.value)
+
+
+def moepp_stack_backward_workspace_bytes(cfg: Config, n_layers: int) -> int:
+    n = ctypes.c_size_t(0)
+    c = cfg.c()
+    _check(lib().moepp_stack_backward_workspace_bytes(ctypes.byref(c), ctypes.c_int32(n_layers), ctypes.byref(n)),
+           "moepp_stack_backward_workspace_bytes")
+    return int(n.value)
+
+
+def moepp_stack_forward_train(cfg, weights_list, x, prev_logits, y, logits_out, workspace):
+    c, arr = cfg.c(), _weights_array(weights_list)
+    _check(lib().moepp_stack_forward_train(ctypes.byref(c), arr, ctypes.c_int32(len(weights_list)), _p(x),
+                                           _p(prev_logits), _p(y), _p(logits_out), _p(workspace),
+                                           ctypes.c_size_t(workspace.numel() * workspace.element_size()), _stream()),
+           "moepp_stack_forward_train")
+
+
+def moepp_stack_backward(cfg, weights_list, x, prev_logits, dy, dlogits_last, balance_scale, balance_loss_out,
+                         train_workspace, grads_list, bwd_workspace):
+    """grads_list: one dict per layer (fields of moepp_grads); dx / dprev are read from the first only."""
+    c, arr = cfg.c(), _weights_array(weights_list)
+    garr = (moepp_grads * len(grads_list))()
+    for i, g in enumerate(grads_list):
+        garr[i] = _grads(g)
+    nbytes = lambda t: ctypes.c_size_t(t.numel() * t.element_size())
+    _check(lib().moepp_stack_backward(ctypes.byref(c), arr, ctypes.c_int32(len(weights_list)), _p(x), _p(prev_logits),
+                                      _p(dy), _p(dlogits_last), ctypes.c_float(balance_scale), _p(balance_loss_out),
+                                      _p(train_workspace), nbytes(train_workspace), garr, _p(bwd_workspace),
+                                      nbytes(bwd_workspace), _stream()), "moepp_stack_backward")
 
 
 def moepp_balance_backward(cfg, logits, f, scale, dlogits, accumulate=False):

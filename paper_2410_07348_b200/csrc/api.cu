@@ -594,31 +594,21 @@ moepp_status moepp_backward_workspace_bytes(const moepp_config* cfg, size_t* byt
   return MOEPP_OK;
 }
 
-moepp_status moepp_layer_backward(const moepp_config* cfg, const moepp_weights* weights, const void* x,
-                                  const float* prev_logits, const float* logits, const void* dy,
-                                  const float* dlogits_next, const void* fwd_workspace, size_t fwd_workspace_bytes,
-                                  const moepp_grads* grads, void* bwd_workspace, size_t bwd_workspace_bytes,
-                                  void* stream) {
-  Dims d;
-  moepp_status s = make_dims(cfg, &d);
+// One layer's backward pass on validated dimensions: argument checks for the gradient set, then the launches.
+static moepp_status layer_backward_on_device(const Dims& d, const moepp_weights* weights, const void* x,
+                                             const float* prev_logits, const float* logits, const void* dy,
+                                             const float* dlogits_next, const char* fw, const moepp_grads& g, char* bw,
+                                             cudaStream_t st) {
+  const moepp_status s = check_layer_args(d, weights, x, prev_logits, dy, fw);
   if (s != MOEPP_OK) return s;
-  if (grads == nullptr || bwd_workspace == nullptr) return MOEPP_ERR_INVALID_ARG;
-  if (d.flags & MOEPP_FLAG_FUSED_GATHER) return MOEPP_ERR_INVALID_ARG;
-  s = check_layer_args(d, weights, x, prev_logits, dy, fwd_workspace);
-  if (s != MOEPP_OK) return s;
-  const moepp_grads& g = *grads;
   if (g.dW_r == nullptr || (d.T > 0 && g.dx == nullptr)) return MOEPP_ERR_INVALID_ARG;
   if (d.T > 0 && weights->W_g != nullptr && g.dprev == nullptr) return MOEPP_ERR_INVALID_ARG;
   if (d.n_const > 0 && (g.dW_c == nullptr || g.dv == nullptr)) return MOEPP_ERR_INVALID_ARG;
   if (d.n_ffn > 0 && (g.dW_gate == nullptr || g.dW_up == nullptr || g.dW_down == nullptr))
     return MOEPP_ERR_INVALID_ARG;
   if (!aligned16(dy) || !aligned16(g.dx) || !aligned16(x)) return MOEPP_ERR_ALIGN;
-  if ((reinterpret_cast<uintptr_t>(bwd_workspace) & (kAlign - 1)) != 0) return MOEPP_ERR_ALIGN;
   const Carve c = carve(d, false);
   const BwdCarve bc = carve_backward(d);
-  if (fwd_workspace_bytes < c.total || bwd_workspace_bytes < bc.total) return MOEPP_ERR_WORKSPACE;
-  const char* fw = static_cast<const char*>(fwd_workspace);
-  char* bw = static_cast<char*>(bwd_workspace);
   ForwardState fs{};
   fs.logits = logits != nullptr ? logits : reinterpret_cast<const float*>(fw + c.logits);
   fs.topk_idx = reinterpret_cast<const int32_t*>(fw + c.topk_idx);
@@ -640,8 +630,169 @@ moepp_status moepp_layer_backward(const moepp_config* cfg, const moepp_weights* 
   b.cx = reinterpret_cast<float*>(bw + bc.cx);
   b.cvq = reinterpret_cast<float*>(bw + bc.cvq);
   b.part = reinterpret_cast<float*>(bw + bc.part);
-  return from_cuda(launch_layer_backward(d, fs, *weights, x, prev_logits, dy, dlogits_next, b, g,
-                                         static_cast<cudaStream_t>(stream)));
+  return from_cuda(launch_layer_backward(d, fs, *weights, x, prev_logits, dy, dlogits_next, b, g, st));
+}
+
+moepp_status moepp_layer_backward(const moepp_config* cfg, const moepp_weights* weights, const void* x,
+                                  const float* prev_logits, const float* logits, const void* dy,
+                                  const float* dlogits_next, const void* fwd_workspace, size_t fwd_workspace_bytes,
+                                  const moepp_grads* grads, void* bwd_workspace, size_t bwd_workspace_bytes,
+                                  void* stream) {
+  Dims d;
+  const moepp_status s = make_dims(cfg, &d);
+  if (s != MOEPP_OK) return s;
+  if (grads == nullptr || bwd_workspace == nullptr) return MOEPP_ERR_INVALID_ARG;
+  if (d.flags & MOEPP_FLAG_FUSED_GATHER) return MOEPP_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(bwd_workspace) & (kAlign - 1)) != 0) return MOEPP_ERR_ALIGN;
+  if (fwd_workspace_bytes < carve(d, false).total || bwd_workspace_bytes < carve_backward(d).total)
+    return MOEPP_ERR_WORKSPACE;
+  return layer_backward_on_device(d, weights, x, prev_logits, logits, dy, dlogits_next,
+                                  static_cast<const char*>(fwd_workspace), *grads, static_cast<char*>(bwd_workspace),
+                                  static_cast<cudaStream_t>(stream));
+}
+
+// ---- a stack that can be differentiated: every layer keeps its own workspace, output and logits ------------
+// slot j = [layer workspace | y of layer j | logits of layer j]
+static size_t train_slot_bytes(const Dims& d, size_t* act, size_t* lg) {
+  stack_extra_bytes(d, act, lg);
+  return carve(d, false).total + *act + *lg;
+}
+
+moepp_status moepp_stack_train_workspace_bytes(const moepp_config* cfg, int32_t n_layers, size_t* bytes) {
+  Dims d;
+  const moepp_status s = make_dims(cfg, &d);
+  if (s != MOEPP_OK) return s;
+  if (bytes == nullptr || n_layers < 1) return MOEPP_ERR_INVALID_ARG;
+  size_t act, lg;
+  *bytes = (size_t)n_layers * train_slot_bytes(d, &act, &lg);
+  return MOEPP_OK;
+}
+
+moepp_status moepp_stack_forward_train(const moepp_config* cfg, const moepp_weights* layers, int32_t n_layers,
+                                       const void* x, const float* prev_logits, void* y, float* logits_out,
+                                       void* workspace, size_t workspace_bytes, void* stream) {
+  Dims d;
+  const moepp_status s = make_dims(cfg, &d);
+  if (s != MOEPP_OK) return s;
+  if (layers == nullptr || n_layers < 1 || workspace == nullptr) return MOEPP_ERR_INVALID_ARG;
+  if (d.T > 0 && (x == nullptr || y == nullptr)) return MOEPP_ERR_INVALID_ARG;
+  if (d.flags & MOEPP_FLAG_FUSED_GATHER) return MOEPP_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(y)) return MOEPP_ERR_ALIGN;
+  if ((reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) != 0) return MOEPP_ERR_ALIGN;
+  size_t act, lg;
+  const size_t slot = train_slot_bytes(d, &act, &lg);
+  if (workspace_bytes < (size_t)n_layers * slot) return MOEPP_ERR_WORKSPACE;
+  if (d.T > 0 && layers[0].W_g != nullptr && prev_logits == nullptr) return MOEPP_ERR_INVALID_ARG;
+  const Carve c = carve(d, false);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char* ws = static_cast<char*>(workspace);
+  const void* cur_x = x;
+  const float* cur_prev = prev_logits;
+  for (int j = 0; j < n_layers; ++j) {
+    char* sl = ws + (size_t)j * slot;
+    const bool last = (j == n_layers - 1);
+    void* out_y = last ? y : static_cast<void*>(sl + c.total);
+    float* out_l = reinterpret_cast<float*>(sl + c.total + act);
+    const moepp_weights* w = &layers[j];
+    const float* prev = (w->W_g != nullptr) ? cur_prev : nullptr;
+    moepp_status r = check_layer_args(d, w, cur_x, prev, out_y, sl);
+    if (r != MOEPP_OK) return r;
+    r = layer_on_device(d, c, w, cur_x, prev, out_y, out_l, sl, st);
+    if (r != MOEPP_OK) return r;
+    cur_x = out_y;
+    cur_prev = out_l;
+  }
+  if (logits_out != nullptr && d.T > 0 &&
+      cudaMemcpyAsync(logits_out, cur_prev, sizeof(float) * (size_t)d.T * d.N, cudaMemcpyDeviceToDevice, st) !=
+          cudaSuccess)
+    return MOEPP_ERR_CUDA;
+  return MOEPP_OK;
+}
+
+// backward scratch of a stack: one layer's scratch, two dx and two dlogits buffers to ping-pong between layers,
+// and the Eq. 7 statistics of the layer in hand (f, P, loss)
+static size_t stack_backward_bytes(const Dims& d, size_t* act, size_t* lg, size_t* stats) {
+  stack_extra_bytes(d, act, lg);
+  *stats = align_up(sizeof(float) * (2 * (size_t)d.N + 1));
+  return carve_backward(d).total + 2 * (*act) + 2 * (*lg) + *stats;
+}
+
+moepp_status moepp_stack_backward_workspace_bytes(const moepp_config* cfg, int32_t n_layers, size_t* bytes) {
+  Dims d;
+  const moepp_status s = make_dims(cfg, &d);
+  if (s != MOEPP_OK) return s;
+  if (bytes == nullptr || n_layers < 1) return MOEPP_ERR_INVALID_ARG;
+  size_t act, lg, stats;
+  *bytes = stack_backward_bytes(d, &act, &lg, &stats);
+  return MOEPP_OK;
+}
+
+moepp_status moepp_stack_backward(const moepp_config* cfg, const moepp_weights* layers, int32_t n_layers, const void* x,
+                                  const float* prev_logits, const void* dy, const float* dlogits_last,
+                                  float balance_scale, float* balance_loss_out, const void* train_workspace,
+                                  size_t train_workspace_bytes, const moepp_grads* grads, void* bwd_workspace,
+                                  size_t bwd_workspace_bytes, void* stream) {
+  Dims d;
+  const moepp_status s = make_dims(cfg, &d);
+  if (s != MOEPP_OK) return s;
+  if (layers == nullptr || grads == nullptr || n_layers < 1 || train_workspace == nullptr || bwd_workspace == nullptr)
+    return MOEPP_ERR_INVALID_ARG;
+  if (d.flags & MOEPP_FLAG_FUSED_GATHER) return MOEPP_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(train_workspace) & (kAlign - 1)) != 0 ||
+      (reinterpret_cast<uintptr_t>(bwd_workspace) & (kAlign - 1)) != 0)
+    return MOEPP_ERR_ALIGN;
+  size_t act, lg, stats;
+  const size_t slot = train_slot_bytes(d, &act, &lg);
+  if (train_workspace_bytes < (size_t)n_layers * slot) return MOEPP_ERR_WORKSPACE;
+  if (bwd_workspace_bytes < stack_backward_bytes(d, &act, &lg, &stats)) return MOEPP_ERR_WORKSPACE;
+  const Carve c = carve(d, false);
+  const size_t bc_total = carve_backward(d).total;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const char* ws = static_cast<const char*>(train_workspace);
+  char* bw = static_cast<char*>(bwd_workspace);
+  void* dxbuf[2] = {bw + bc_total, bw + bc_total + act};
+  float* dlbuf[2] = {reinterpret_cast<float*>(bw + bc_total + 2 * act),
+                     reinterpret_cast<float*>(bw + bc_total + 2 * act + lg)};
+  float* st_f = reinterpret_cast<float*>(bw + bc_total + 2 * act + 2 * lg);
+  float* st_P = st_f + d.N;
+  float* st_loss = st_P + d.N;
+  const size_t lg_bytes = sizeof(float) * (size_t)d.T * d.N;
+  const bool balance = balance_scale != 0.f;
+
+  for (int j = n_layers - 1; j >= 0; --j) {
+    const char* sl = ws + (size_t)j * slot;
+    const moepp_weights* w = &layers[j];
+    const bool last = (j == n_layers - 1);
+    const void* x_j = j == 0 ? x : static_cast<const void*>(ws + (size_t)(j - 1) * slot + c.total);
+    const float* in_logits = j == 0 ? prev_logits : reinterpret_cast<const float*>(ws + (size_t)(j - 1) * slot + c.total + act);
+    const float* prev_j = (w->W_g != nullptr) ? in_logits : nullptr;
+    const float* logits_j = reinterpret_cast<const float*>(sl + c.total + act);
+    const void* dy_j = last ? dy : dxbuf[(j + 1) & 1];
+    // what arrives at this layer's logits from above: the next layer's dprev, or the caller's dlogits_last
+    const float* dl = last ? dlogits_last : (layers[j + 1].W_g != nullptr ? dlbuf[(j + 1) & 1] : nullptr);
+    if (balance && d.T > 0) {  // + balance_scale * dL_b/dlogits of this layer (Eq. 7)
+      const int32_t* counts = reinterpret_cast<const int32_t*>(sl + c.counts);
+      if (launch_balance_stats(d, logits_j, counts, st_f, st_P, st_loss, st) != cudaSuccess) return MOEPP_ERR_CUDA;
+      if (balance_loss_out != nullptr &&
+          cudaMemcpyAsync(balance_loss_out + j, st_loss, sizeof(float), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+        return MOEPP_ERR_CUDA;
+      float* mine = dlbuf[(j + 1) & 1];
+      if (last && dl != nullptr) {
+        if (cudaMemcpyAsync(mine, dl, lg_bytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return MOEPP_ERR_CUDA;
+      }
+      if (launch_balance_backward(d, logits_j, st_f, balance_scale, dl != nullptr ? 1 : 0, mine, st) != cudaSuccess)
+        return MOEPP_ERR_CUDA;
+      dl = mine;
+    }
+    moepp_grads g = grads[j];
+    if (j > 0) {
+      g.dx = dxbuf[j & 1];
+      g.dprev = (w->W_g != nullptr) ? dlbuf[j & 1] : nullptr;
+    }
+    const moepp_status r = layer_backward_on_device(d, w, x_j, prev_j, logits_j, dy_j, dl, sl, g, bw, st);
+    if (r != MOEPP_OK) return r;
+  }
+  return MOEPP_OK;
 }
 
 moepp_status moepp_device_error(int32_t* code) {
