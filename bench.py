@@ -390,6 +390,33 @@ def main():
                "recomputed_pre_activations": fwd_bwd(args.flags, 16.0)}
         del grads
 
+        # whole stack, forward (every layer keeps its state) + backward with the Eq. 7 gradient of every layer
+        cfg_t = B.config_from_spec(spec, add_residual=add_res, flags=args.flags | B.FLAG_SAVE_PREACT, tau=args.tau,
+                                   capacity_factor=args.capacity_factor, row_align=64)
+        tws = torch.empty(B.moepp_stack_train_workspace_bytes(cfg_t, L), dtype=torch.uint8, device=dev)
+        sbw = torch.empty(B.moepp_stack_backward_workspace_bytes(cfg_t, L), dtype=torch.uint8, device=dev)
+        glist = []
+        for wl in wds:
+            has_g = wl["W_g"] is not None
+            glist.append(dict(dx=torch.empty_like(x0), dprev=fz(T, N), dW_r=fz(N, spec.D), dW_g=fz(N, N) if has_g else None,
+                              dbias=fz(N), dW_c=fz(max(spec.n_const, 1), 2, spec.D), dv=fz(max(spec.n_const, 1), spec.D),
+                              dW_gate=fz(spec.n_ffn, spec.F, spec.D), dW_up=fz(spec.n_ffn, spec.F, spec.D),
+                              dW_down=fz(spec.n_ffn, spec.D, spec.F)))
+        lb = fz(L)
+        p_in = prev0 if wds[0]["W_g"] is not None else None
+
+        def train_step():
+            B.moepp_stack_forward_train(cfg_t, wds, x0, p_in, y_out, lg_out, tws)
+            B.moepp_stack_backward(cfg_t, wds, x0, p_in, dy, None, 0.01, lb, tws, glist, sbw)
+
+        ms_train, _ = timed(train_step, max(3, args.steps // 5), 3)
+        assert B.moepp_device_error() == 0
+        bwd["train_step"] = {"what": "%d layers: moepp_stack_forward_train + moepp_stack_backward (all gradients, "
+                                     "beta = 0.01 times every layer's Eq. 7 gradient), kept pre-activations" % L,
+                             "ms_per_step": ms_train, "tokens_per_s": world * T * L / (ms_train * 1e-3),
+                             "balance_loss_per_layer": [float(v) for v in lb.cpu()]}
+        del tws, sbw, glist
+
     # ---- end to end through the host-buffer call --------------------------------------------------------------
     xh = x0.cpu().pin_memory()
     yh = torch.empty(T, spec.D, dtype=td).pin_memory()

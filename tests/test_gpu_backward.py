@@ -202,6 +202,14 @@ def test_backward_through_two_chained_layers(oracle64):
             assert err <= 5e-4, (name, err)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_backward_at_the_expert_count_limits(oracle64, dtype):
+    """N = 64 experts, 16 of them constant experts (96 router rows), top-8: the widest tables every kernel takes."""
+    spec = W.LayerSpec(T=700, D=264, F=72, n_ffn=40, n_zero=4, n_copy=4, n_const=16, top_k=8, dtype=dtype)
+    lt = W.make_layer(spec, seed=13, with_prev=True, w_std=0.05)
+    check_backward(oracle64, lt, row_align=64, renorm_topk=1, add_residual=1)
+
+
 def test_backward_no_tokens():
     spec = W.LayerSpec(T=0, D=64, F=96, n_ffn=2, n_zero=1, n_copy=1, n_const=1, top_k=2, dtype="f32")
     lt = W.make_layer(spec, seed=0, with_prev=True)
