@@ -210,6 +210,47 @@ def test_backward_at_the_expert_count_limits(oracle64, dtype):
     check_backward(oracle64, lt, row_align=64, renorm_topk=1, add_residual=1)
 
 
+def test_backward_full_size_layer_on_sampled_tokens(oracle64):
+    """The benchmark's layer shape and launch configuration (T = 32768, d_model 4096, d_ffn 2816, 16 + 4 experts, bf16,
+    64-row segments, kept pre-activations).  dy and dlogits are non-zero on 20 sampled tokens only, so every gradient
+    is the sum of those tokens' contributions, which the oracle computes from the 20-token sub-batch (tokens are
+    independent without a capacity limit); all other tokens must get an exactly zero dx."""
+    spec = W.CONFIGS["cfg4_7b_stack"]
+    lt = W.make_layer(spec, seed=1, with_prev=True, w_std=0.02, device="cuda", gen_device="cuda")
+    cfg = B.config_from_spec(spec, add_residual=1, row_align=64, flags=B.FLAG_SAVE_PREACT)
+    wd = B.weights_from_tensors(lt)
+    n_tok = 20
+    rng = np.random.default_rng(4)
+    toks = np.sort(rng.choice(spec.T, n_tok, replace=False))
+    gen = torch.Generator().manual_seed(44)
+    dy_s = torch.randn(n_tok, spec.D, generator=gen).to(torch.bfloat16)
+    dl_s = 0.1 * torch.randn(n_tok, spec.N, generator=gen)
+    dy = torch.zeros(spec.T, spec.D, dtype=torch.bfloat16, device="cuda")
+    dl = torch.zeros(spec.T, spec.N, device="cuda")
+    tk = torch.as_tensor(toks, device="cuda")
+    dy[tk] = dy_s.cuda()
+    dl[tk] = dl_s.cuda()
+    got, idx_g = gpu_backward(cfg, wd, lt.x, lt.prev, dy, dl)
+
+    sub = W.LayerSpec(n_tok, spec.D, spec.F, spec.n_ffn, spec.n_zero, spec.n_copy, spec.n_const, spec.top_k, "bf16")
+    s = shape_of(sub, add_residual=1, row_align=64)
+    x_s, prev_s = f32(lt.x[tk]), f32(lt.prev[tk])
+    lt.x, lt.prev = None, None
+    oi = oracle_inputs(lt)
+    ref = oracle64.layer_backward(s, x_s, oi["W_r"], idx_g[toks], f32(dy_s), oi["W_g"], prev_s, oi["bias"], oi["W_c"],
+                                  oi["v"], f32(lt.W_gate), f32(lt.W_up), f32(lt.W_down), dlogits=f32(dl_s))
+    for name in GRADS:
+        r, g = ref[name], got[name]
+        if name in ("dx", "dprev"):
+            rest = np.ones(spec.T, bool)
+            rest[toks] = False
+            assert not np.any(g[rest]), name  # untouched tokens: exact zeros
+            g = g[toks]
+        scale = max(float(np.abs(r).max()), 1e-6)
+        err = float(np.abs(g.reshape(r.shape).astype(np.float64) - r).max()) / scale
+        assert err <= TOL["bf16"], (name, err)
+
+
 def test_backward_no_tokens():
     spec = W.LayerSpec(T=0, D=64, F=96, n_ffn=2, n_zero=1, n_copy=1, n_const=1, top_k=2, dtype="f32")
     lt = W.make_layer(spec, seed=0, with_prev=True)
