@@ -280,7 +280,7 @@ constexpr int kDxGroups = 4;   // groups of 32 tokens a block serves one after t
 // staged in shared memory once; the block then serves four groups of 32 tokens, each warp kDxTokens of them, a lane
 // holding columns 4 lane .. 4 lane + 3 and 128 + 4 lane .. of the slab (conflict-free 16-byte shared loads).
 template <typename XT>
-__global__ void __launch_bounds__(kWarpsPerBlock * 32, 3)
+__global__ void __launch_bounds__(kWarpsPerBlock * 32, 2)
 dx_assemble_kernel(Dims dm, int R, const XT* __restrict__ dy, const float* __restrict__ cx,
                    const float* __restrict__ dGz, const float* __restrict__ W_r, const float* __restrict__ W_c,
                    const XT* __restrict__ dXp, const int32_t* __restrict__ topk_idx,
@@ -299,6 +299,21 @@ dx_assemble_kernel(Dims dm, int R, const XT* __restrict__ dy, const float* __res
       v = __ldg(reinterpret_cast<const float4*>(wrow + d0 + c4));
     }
     *reinterpret_cast<float4*>(s_w + (size_t)r * kDxSlab + c4) = v;
+  }
+  // rows of the first two picks and cx of every token this warp will serve (all groups), fetched up front
+  __shared__ int s_rows[kWarpsPerBlock][kDxGroups * kDxTokens * 2];
+  __shared__ float s_cx[kWarpsPerBlock][kDxGroups * kDxTokens];
+  {
+    const int grp = lane / (kDxTokens * 2), j = (lane / 2) % kDxTokens, k = lane & 1;
+    const long long t = (((long long)blockIdx.x * kDxGroups + grp) * kWarpsPerBlock + wib) * kDxTokens + j;
+    int row = -1;
+    if (grp < kDxGroups && t < dm.T && k < K && topk_idx[t * K + k] < dm.n_ffn) row = row_of_slot[t * K + k];  // -2: dropped
+    if (grp < kDxGroups) s_rows[wib][lane] = row;
+    if (lane < kDxGroups * kDxTokens) {
+      const long long tc = (((long long)blockIdx.x * kDxGroups + lane / kDxTokens) * kWarpsPerBlock + wib) * kDxTokens +
+                           lane % kDxTokens;
+      s_cx[wib][lane] = tc < dm.T ? cx[tc] : 0.f;
+    }
   }
   __syncthreads();
   // the two 4-column groups of this lane
@@ -323,29 +338,51 @@ dx_assemble_kernel(Dims dm, int R, const XT* __restrict__ dy, const float* __res
       s_c[i] = j < nt ? dGz[(t0 + j) * R + r] : 0.f;
     }
     __syncwarp();
-    // accumulators start from cx dy + the grouped rows of the kept FFN picks
+    // cx dy + the grouped rows of the kept FFN picks.  16-bit storage: the rows of dy and of the first two picks are
+    // requested here as raw words and only unpacked after the weight loop, which covers their latency.
+    constexpr bool kEarly = sizeof(XT) == 2;
+    uint2 ra[kDxTokens][3], rb[kDxTokens][3];
     float acc[kDxTokens][8];
 #pragma unroll
     for (int j = 0; j < kDxTokens; ++j) {
 #pragma unroll
       for (int i = 0; i < 8; ++i) acc[j][i] = 0.f;
-      if (j < nt) {
-        const float c = cx[t0 + j];
-        float va[4] = {0.f, 0.f, 0.f, 0.f}, vb[4] = {0.f, 0.f, 0.f, 0.f};
-        const XT* src = dy + (size_t)(t0 + j) * D;
-        if (a_ok) load4(src + ca, va);
-        if (b_ok) load4(src + cb, vb);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) { acc[j][i] = c * va[i]; acc[j][4 + i] = c * vb[i]; }
-        for (int k = 0; k < K; ++k) {
-          if (topk_idx[(t0 + j) * K + k] >= dm.n_ffn) continue;
-          const int row = row_of_slot[(t0 + j) * K + k];  // -2: dropped
-          if (row < 0) continue;
-          src = dXp + (size_t)row * D;
+      for (int k = 0; k < 3; ++k) ra[j][k] = rb[j][k] = make_uint2(0u, 0u);  // bf16 zeros
+      if (j < nt) {
+        const int r0 = s_rows[wib][(grp * kDxTokens + j) * 2], r1 = s_rows[wib][(grp * kDxTokens + j) * 2 + 1];
+        if (kEarly) {
+          const XT* src = dy + (size_t)(t0 + j) * D;
+          if (a_ok) ra[j][0] = *reinterpret_cast<const uint2*>(src + ca);
+          if (b_ok) rb[j][0] = *reinterpret_cast<const uint2*>(src + cb);
+          if (r0 >= 0) {
+            src = dXp + (size_t)r0 * D;
+            if (a_ok) ra[j][1] = *reinterpret_cast<const uint2*>(src + ca);
+            if (b_ok) rb[j][1] = *reinterpret_cast<const uint2*>(src + cb);
+          }
+          if (r1 >= 0) {
+            src = dXp + (size_t)r1 * D;
+            if (a_ok) ra[j][2] = *reinterpret_cast<const uint2*>(src + ca);
+            if (b_ok) rb[j][2] = *reinterpret_cast<const uint2*>(src + cb);
+          }
+        } else {
+          const float c = s_cx[wib][grp * kDxTokens + j];
+          float va[4] = {0.f, 0.f, 0.f, 0.f}, vb[4] = {0.f, 0.f, 0.f, 0.f};
+          const XT* src = dy + (size_t)(t0 + j) * D;
           if (a_ok) load4(src + ca, va);
           if (b_ok) load4(src + cb, vb);
 #pragma unroll
-          for (int i = 0; i < 4; ++i) { if (a_ok) acc[j][i] += va[i]; if (b_ok) acc[j][4 + i] += vb[i]; }
+          for (int i = 0; i < 4; ++i) { acc[j][i] = c * va[i]; acc[j][4 + i] = c * vb[i]; }
+#pragma unroll
+          for (int k = 0; k < 2; ++k) {
+            const int row = k ? r1 : r0;
+            if (row < 0) continue;
+            src = dXp + (size_t)row * D;
+            if (a_ok) load4(src + ca, va);
+            if (b_ok) load4(src + cb, vb);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { if (a_ok) acc[j][i] += va[i]; if (b_ok) acc[j][4 + i] += vb[i]; }
+          }
         }
       }
     }
@@ -364,6 +401,28 @@ dx_assemble_kernel(Dims dm, int R, const XT* __restrict__ dy, const float* __res
 #pragma unroll
     for (int j = 0; j < kDxTokens; ++j) {
       if (j >= nt) continue;
+      if (kEarly) {
+        const float c = s_cx[wib][grp * kDxTokens + j];
+        acc[j][0] += fmaf(c, bf16_lo(ra[j][0].x), bf16_lo(ra[j][1].x) + bf16_lo(ra[j][2].x));
+        acc[j][1] += fmaf(c, bf16_hi(ra[j][0].x), bf16_hi(ra[j][1].x) + bf16_hi(ra[j][2].x));
+        acc[j][2] += fmaf(c, bf16_lo(ra[j][0].y), bf16_lo(ra[j][1].y) + bf16_lo(ra[j][2].y));
+        acc[j][3] += fmaf(c, bf16_hi(ra[j][0].y), bf16_hi(ra[j][1].y) + bf16_hi(ra[j][2].y));
+        acc[j][4] += fmaf(c, bf16_lo(rb[j][0].x), bf16_lo(rb[j][1].x) + bf16_lo(rb[j][2].x));
+        acc[j][5] += fmaf(c, bf16_hi(rb[j][0].x), bf16_hi(rb[j][1].x) + bf16_hi(rb[j][2].x));
+        acc[j][6] += fmaf(c, bf16_lo(rb[j][0].y), bf16_lo(rb[j][1].y) + bf16_lo(rb[j][2].y));
+        acc[j][7] += fmaf(c, bf16_hi(rb[j][0].y), bf16_hi(rb[j][1].y) + bf16_hi(rb[j][2].y));
+      }
+      for (int k = 2; k < K; ++k) {  // picks beyond the second
+        if (topk_idx[(t0 + j) * K + k] >= dm.n_ffn) continue;
+        const int row = row_of_slot[(t0 + j) * K + k];  // -2: dropped
+        if (row < 0) continue;
+        float va[4] = {0.f, 0.f, 0.f, 0.f}, vb[4] = {0.f, 0.f, 0.f, 0.f};
+        const XT* src = dXp + (size_t)row * D;
+        if (a_ok) load4(src + ca, va);
+        if (b_ok) load4(src + cb, vb);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { acc[j][i] += va[i]; acc[j][4 + i] += vb[i]; }
+      }
       XT* dst = dx + (size_t)(t0 + j) * D;
       if (sizeof(XT) == 2) {
         if (a_ok) *reinterpret_cast<uint2*>(dst + ca) = make_uint2(pack_bf16(acc[j][0], acc[j][1]), pack_bf16(acc[j][2], acc[j][3]));
@@ -386,14 +445,36 @@ __global__ void __launch_bounds__(kOuterThreads)
 token_outer_rows_kernel(const float* __restrict__ A, const TB* __restrict__ B, float* __restrict__ part, int T, int M,
                         int Nout, long long a_rs, long long b_rs, int chunk) {
   constexpr int TS = 32;  // tokens staged per trip
+  constexpr int G = 8;    // tokens per group of loads in flight
+  constexpr int W4 = sizeof(TB) == 2 ? 2 : 4;  // 32-bit words per 4 elements of B
   __shared__ __align__(16) float s_a[TS][RT];
   const int z = blockIdx.y, n = (blockIdx.x * kOuterThreads + threadIdx.x) * 4;
   const int t_begin = z * chunk, t_end = min(T, t_begin + chunk);
   const bool col_ok = n < Nout;  // Nout is a multiple of 4
+  // raw words of B for one group of G tokens; the next group is requested before the current one is used
+  auto fetch = [&](int t0, uint32_t (&raw)[G][W4]) {
+#pragma unroll
+    for (int j = 0; j < G; ++j) {
+#pragma unroll
+      for (int w = 0; w < W4; ++w) raw[j][w] = 0u;
+      if (col_ok && t0 + j < t_end) {
+        const TB* bp = B + (size_t)(t0 + j) * b_rs + n;
+        if (W4 == 2) {
+          const uint2 u = *reinterpret_cast<const uint2*>(bp);
+          raw[j][0] = u.x; raw[j][1] = u.y;
+        } else {
+          const uint4 u = *reinterpret_cast<const uint4*>(bp);
+          raw[j][0] = u.x; raw[j][1] = u.y; raw[j][W4 - 2] = u.z; raw[j][W4 - 1] = u.w;
+        }
+      }
+    }
+  };
   for (int m0 = 0; m0 < M; m0 += RT) {
     float acc[RT][4];
 #pragma unroll
     for (int r = 0; r < RT; ++r) acc[r][0] = acc[r][1] = acc[r][2] = acc[r][3] = 0.f;
+    uint32_t cur[G][W4], nxt[G][W4];
+    fetch(t_begin, cur);
     for (int ts = t_begin; ts < t_end; ts += TS) {
       __syncthreads();
       for (int i = threadIdx.x; i < TS * RT; i += kOuterThreads) {
@@ -401,37 +482,32 @@ token_outer_rows_kernel(const float* __restrict__ A, const TB* __restrict__ B, f
         s_a[tt][r] = (ts + tt < t_end && m0 + r < M) ? A[(size_t)(ts + tt) * a_rs + m0 + r] : 0.f;
       }
       __syncthreads();
-      if (col_ok) {
+#pragma unroll 1
+      for (int t8 = 0; t8 < TS; t8 += G) {  // not unrolled: the body is already several hundred FMAs
+        fetch(ts + t8 + G, nxt);  // may reach into the next trip; beyond t_end it fetches nothing
 #pragma unroll
-        for (int t8 = 0; t8 < TS; t8 += 8) {
-          float bv[8][4];
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {  // eight independent loads in flight
-            bv[j][0] = bv[j][1] = bv[j][2] = bv[j][3] = 0.f;
-            if (ts + t8 + j < t_end) {
-              const TB* bp = B + (size_t)(ts + t8 + j) * b_rs + n;
-              if (sizeof(TB) == 2) {
-                const uint2 u = *reinterpret_cast<const uint2*>(bp);
-                bv[j][0] = bf16_lo(u.x); bv[j][1] = bf16_hi(u.x); bv[j][2] = bf16_lo(u.y); bv[j][3] = bf16_hi(u.y);
-              } else {
-                const float4 f = *reinterpret_cast<const float4*>(bp);
-                bv[j][0] = f.x; bv[j][1] = f.y; bv[j][2] = f.z; bv[j][3] = f.w;
-              }
-            }
+        for (int j = 0; j < G; ++j) {
+          float bv[4];
+          if (W4 == 2) {
+            bv[0] = bf16_lo(cur[j][0]); bv[1] = bf16_hi(cur[j][0]); bv[2] = bf16_lo(cur[j][1]); bv[3] = bf16_hi(cur[j][1]);
+          } else {
+            bv[0] = __uint_as_float(cur[j][0]); bv[1] = __uint_as_float(cur[j][1]);
+            bv[2] = __uint_as_float(cur[j][W4 - 2]); bv[3] = __uint_as_float(cur[j][W4 - 1]);
           }
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
+          for (int r4 = 0; r4 < RT; r4 += 4) {
+            const float4 av = *reinterpret_cast<const float4*>(&s_a[t8 + j][r4]);
+            const float ar[4] = {av.x, av.y, av.z, av.w};
 #pragma unroll
-            for (int r4 = 0; r4 < RT; r4 += 4) {
-              const float4 av = *reinterpret_cast<const float4*>(&s_a[t8 + j][r4]);
-              const float ar[4] = {av.x, av.y, av.z, av.w};
+            for (int r = 0; r < 4; ++r)
 #pragma unroll
-              for (int r = 0; r < 4; ++r)
-#pragma unroll
-                for (int i = 0; i < 4; ++i) acc[r4 + r][i] = fmaf(ar[r], bv[j][i], acc[r4 + r][i]);
-            }
+              for (int i = 0; i < 4; ++i) acc[r4 + r][i] = fmaf(ar[r], bv[i], acc[r4 + r][i]);
           }
         }
+#pragma unroll
+        for (int j = 0; j < G; ++j)
+#pragma unroll
+          for (int w = 0; w < W4; ++w) cur[j][w] = nxt[j][w];
       }
     }
     if (col_ok) {
@@ -446,11 +522,14 @@ token_outer_rows_kernel(const float* __restrict__ A, const TB* __restrict__ B, f
 
 }  // namespace
 
-// The reductions over tokens run in at most 128 chunks of at least 256 tokens.
+// Chunks of the reductions over tokens: enough of them that, with D / 512 column blocks each, about 900 CTAs are
+// in the grid (two rounds of three CTAs per SM), but no chunk shorter than 64 tokens.
 int backward_token_chunks(const Dims& d, int* chunk_tokens) {
-  int chunk = (d.T + 127) / 128;
-  if (chunk < 256) chunk = 256;
-  chunk = (chunk + kOk - 1) / kOk * kOk;
+  const int col_blocks = (d.D + 511) / 512;
+  const int want = (888 + col_blocks - 1) / col_blocks;
+  int chunk = (d.T + want - 1) / want;
+  if (chunk < 64) chunk = 64;
+  chunk = (chunk + 31) / 32 * 32;
   if (chunk_tokens != nullptr) *chunk_tokens = chunk;
   return d.T > 0 ? (d.T + chunk - 1) / chunk : 1;
 }
