@@ -29,7 +29,9 @@ constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kBoxBytes = 64 * BK * 2; // one 64 x 64 box of an MN-major operand: 8 KiB
 constexpr int kThreads = 192;
 constexpr int kTmemCols = 512;
-constexpr int kSmemBytes = kStages * kStageBytes + 1024;
+constexpr int kStagePitch = 36;  // floats per row of an epilogue warp's 32 x 32 staging piece (conflict-free)
+constexpr int kEpiStageBytes = 4 * 32 * kStagePitch * 4;  // four epilogue warps (used by the DH mode)
+constexpr int kSmemBytes = kStages * kStageBytes + 1024 + kEpiStageBytes;
 
 enum Mode { DH = 0, DX = 1, WGRAD = 2 };
 
@@ -255,32 +257,53 @@ bwd_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant_
         const bool row_ok = grow < ti.row_end;
         const size_t at = (size_t)(row_ok ? grow : 0) * a.Nout + ti.n0;
         if (MODE == DH) {
-          // gate / up of the next 16 columns are fetched while the current 16 are worked on
-          uint4 gq[2], uq[2], gn[2], un[2];
-          auto fetch = [&](int c, uint4 (&g)[2], uint4 (&u)[2]) {
+          // 32 columns at a time: the warp parks its 32 x 32 piece of dH in shared memory (a thread holds a row),
+          // then works on it 8 rows at a time with 4 lanes per row and 8 columns per lane, so that the gate / up
+          // reads and the dGate / dUp writes cover 64 contiguous bytes per row (8 lines per warp instruction instead
+          // of 32).  gate / up of the next 32 columns are requested while the current ones are worked on.
+          float* stage = reinterpret_cast<float*>(smem_raw + (ring - smem_u32(smem_raw)) + kStages * kStageBytes) +
+                         (warp - 2) * (32 * kStagePitch);
+          const int sub_row = lane >> 2, sub_col = (lane & 3) * 8;
+          uint4 gq[4], uq[4], gn[4], un[4];
+          auto fetch = [&](int c, uint4 (&g)[4], uint4 (&u)[4]) {
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
-              g[half] = make_uint4(0u, 0u, 0u, 0u);
-              u[half] = make_uint4(0u, 0u, 0u, 0u);
-              if (row_ok && ti.n0 + c + 8 * half + 8 <= a.Nout) {
-                g[half] = *reinterpret_cast<const uint4*>(a.gate_in + at + c + 8 * half);
-                u[half] = *reinterpret_cast<const uint4*>(a.up_in + at + c + 8 * half);
+            for (int p = 0; p < 4; ++p) {
+              g[p] = make_uint4(0u, 0u, 0u, 0u);
+              u[p] = make_uint4(0u, 0u, 0u, 0u);
+              const int gr = ti.row0 + q * 32 + p * 8 + sub_row;
+              if (gr < ti.row_end && ti.n0 + c + sub_col + 8 <= a.Nout) {
+                const size_t o = (size_t)gr * a.Nout + ti.n0 + c + sub_col;
+                g[p] = *reinterpret_cast<const uint4*>(a.gate_in + o);
+                u[p] = *reinterpret_cast<const uint4*>(a.up_in + o);
               }
             }
           };
           fetch(0, gq, uq);
 #pragma unroll 1
-          for (int c = 0; c < BN; c += 16) {
-            if (c + 16 < BN) fetch(c + 16, gn, un);
-            uint32_t r[16];
-            tmem_ld16(t_row + c, r);
+          for (int c = 0; c < BN; c += 32) {
+            if (c + 32 < BN) fetch(c + 32, gn, un);
+            uint32_t r0[16], r1[16];
+            tmem_ld16(t_row + c, r0);
+            tmem_ld16(t_row + c + 16, r1);
             tmem_ld_wait();
-            tmem_ld_pin(r);
+            tmem_ld_pin(r0);
+            tmem_ld_pin(r1);
+            float* mine = stage + lane * kStagePitch;
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
-              if (!row_ok || ti.n0 + c + 8 * half + 8 > a.Nout) continue;
-              const uint32_t gw[4] = {gq[half].x, gq[half].y, gq[half].z, gq[half].w};
-              const uint32_t uw[4] = {uq[half].x, uq[half].y, uq[half].z, uq[half].w};
+            for (int v = 0; v < 4; ++v) {
+              *reinterpret_cast<uint4*>(mine + 4 * v) = make_uint4(r0[4 * v], r0[4 * v + 1], r0[4 * v + 2], r0[4 * v + 3]);
+              *reinterpret_cast<uint4*>(mine + 16 + 4 * v) = make_uint4(r1[4 * v], r1[4 * v + 1], r1[4 * v + 2], r1[4 * v + 3]);
+            }
+            __syncwarp();
+#pragma unroll
+            for (int p = 0; p < 4; ++p) {
+              const int gr = ti.row0 + q * 32 + p * 8 + sub_row;
+              const float4 d0 = *reinterpret_cast<const float4*>(stage + (p * 8 + sub_row) * kStagePitch + sub_col);
+              const float4 d1 = *reinterpret_cast<const float4*>(stage + (p * 8 + sub_row) * kStagePitch + sub_col + 4);
+              if (gr >= ti.row_end || ti.n0 + c + sub_col + 8 > a.Nout) continue;
+              const float dh[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
+              const uint32_t gw[4] = {gq[p].x, gq[p].y, gq[p].z, gq[p].w};
+              const uint32_t uw[4] = {uq[p].x, uq[p].y, uq[p].z, uq[p].w};
               uint32_t og[4], ou[4];
 #pragma unroll
               for (int i = 0; i < 4; ++i) {
@@ -289,18 +312,20 @@ bwd_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant_
                 for (int j = 0; j < 2; ++j) {
                   const float g = j ? bf16_hi(gw[i]) : bf16_lo(gw[i]);
                   const float u = j ? bf16_hi(uw[i]) : bf16_lo(uw[i]);
-                  const float dh = __uint_as_float(r[8 * half + 2 * i + j]);
                   const float sg = __fdividef(1.f, 1.f + __expf(-g));
-                  dg2[j] = dh * u * (sg + g * sg * (1.f - sg));
-                  du2[j] = dh * g * sg;
+                  dg2[j] = dh[2 * i + j] * u * (sg + g * sg * (1.f - sg));
+                  du2[j] = dh[2 * i + j] * g * sg;
                 }
                 og[i] = pack_bf16(dg2[0], dg2[1]);
                 ou[i] = pack_bf16(du2[0], du2[1]);
               }
-              *reinterpret_cast<uint4*>(a.gate + at + c + 8 * half) = make_uint4(og[0], og[1], og[2], og[3]);
-              *reinterpret_cast<uint4*>(a.up + at + c + 8 * half) = make_uint4(ou[0], ou[1], ou[2], ou[3]);
+              const size_t o = (size_t)gr * a.Nout + ti.n0 + c + sub_col;
+              *reinterpret_cast<uint4*>(a.gate + o) = make_uint4(og[0], og[1], og[2], og[3]);
+              *reinterpret_cast<uint4*>(a.up + o) = make_uint4(ou[0], ou[1], ou[2], ou[3]);
             }
-            gq[0] = gn[0]; gq[1] = gn[1]; uq[0] = un[0]; uq[1] = un[1];
+            __syncwarp();  // the piece is consumed before the next one overwrites it
+#pragma unroll
+            for (int p = 0; p < 4; ++p) { gq[p] = gn[p]; uq[p] = un[p]; }
           }
         } else {
 #pragma unroll 1
