@@ -403,10 +403,13 @@ HostChunks host_chunks(const Dims& d) {
   return h;
 }
 
-Dims chunk_dims(const Dims& d, int tokens) {
+// A chunk holds a fraction of every expert's rows, so the 256-row tiles of the CTA-pair kernels would be padded
+// more heavily: chunks run the 128-row single-CTA kernels (the same arithmetic per element, the same bits).
+Dims chunk_dims(const Dims& d, int tokens, bool chunked) {
   Dims c = d;
   c.T = tokens;
   c.M_cap = (long long)tokens * d.K + (long long)d.n_ffn * (d.row_align - 1);
+  if (chunked && !(d.flags & (MOEPP_FLAG_SAVE_PREACT | MOEPP_FLAG_FUSED_GATHER))) c.flags |= MOEPP_FLAG_FFN_SINGLE_CTA;
   return c;
 }
 
@@ -428,7 +431,7 @@ moepp_status moepp_stack_workspace_bytes_host(const moepp_config* cfg, int32_t n
   size_t total = 0;
   for (int i = 0; i < h.n; ++i) {
     const int tok = (i + 1 < h.n) ? h.tokens : d.T - i * h.tokens;
-    total += chunk_ws_bytes(chunk_dims(d, tok));
+    total += chunk_ws_bytes(chunk_dims(d, tok, h.n > 1));
   }
   *bytes = total;
   return MOEPP_OK;
@@ -482,7 +485,7 @@ moepp_status moepp_stack_forward_host(const moepp_config* cfg, const moepp_weigh
   for (int i = 0; i < h.n && result == MOEPP_OK; ++i) {
     const int t_begin = i * h.tokens;
     const int tok = (i + 1 < h.n) ? h.tokens : d.T - t_begin;
-    const Dims c = chunk_dims(d, tok);
+    const Dims c = chunk_dims(d, tok, h.n > 1);
     size_t act, lg;
     const size_t extra = stack_extra_bytes(c, &act, &lg);
     const size_t base = carve(c, false).total + extra;
