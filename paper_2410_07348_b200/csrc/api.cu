@@ -561,7 +561,7 @@ moepp_status moepp_balance_backward(const moepp_config* cfg, const float* logits
 
 // Device scratch of the backward pass, carved like the forward workspace.
 struct BwdCarve {
-  size_t dYp, gate, up, dXp, dw, dGz, cx, cvq, part, total;
+  size_t dYp, gate, up, dXp, dw, dGz, cx, cvq, part, split, segs, total;
 };
 
 static BwdCarve carve_backward(const Dims& d) {
@@ -582,8 +582,9 @@ static BwdCarve carve_backward(const Dims& d) {
   c.dGz = take(sizeof(float) * (size_t)d.T * R);
   c.cx = take(sizeof(float) * (size_t)d.T);
   c.cvq = take(sizeof(float) * (size_t)d.T * d.n_const);
-  const size_t widest = R * (size_t)d.D > (size_t)d.N * d.N ? R * (size_t)d.D : (size_t)d.N * d.N;
-  c.part = take(sizeof(float) * widest * (size_t)backward_token_chunks(d, nullptr));
+  c.part = take(sizeof(float) * backward_part_floats(d));
+  c.split = take(2 * (size_t)d.T * 128);
+  c.segs = take(sizeof(int32_t) * (kMaxExperts + 1));
   c.total = off;
   return c;
 }
@@ -633,6 +634,8 @@ static moepp_status layer_backward_on_device(const Dims& d, const moepp_weights*
   b.cx = reinterpret_cast<float*>(bw + bc.cx);
   b.cvq = reinterpret_cast<float*>(bw + bc.cvq);
   b.part = reinterpret_cast<float*>(bw + bc.part);
+  b.split = bw + bc.split;
+  b.segs = reinterpret_cast<int32_t*>(bw + bc.segs);
   return from_cuda(launch_layer_backward(d, fs, *weights, x, prev_logits, dy, dlogits_next, b, g, st));
 }
 

@@ -522,6 +522,26 @@ token_outer_rows_kernel(const float* __restrict__ A, const TB* __restrict__ B, f
 
 }  // namespace
 
+// Token segments of the tensor-core reductions: about four 128 x 256 tiles per SM in the grid, whole 64-token k
+// tiles per segment, at most 64 segments (the kernel's segment table).
+int backward_token_segments(const Dims& d, int* tokens_per_segment) {
+  const int n_tiles = (d.D + 255) / 256;
+  int want = (592 + n_tiles - 1) / n_tiles;
+  if (want > 64) want = 64;
+  int per = ((d.T + want - 1) / want + 63) / 64 * 64;
+  if (per < 64) per = 64;
+  if (tokens_per_segment != nullptr) *tokens_per_segment = per;
+  return d.T > 0 ? (d.T + per - 1) / per : 1;
+}
+
+size_t backward_part_floats(const Dims& d) {
+  const size_t R = (size_t)d.N + 2 * (size_t)d.n_const;
+  const size_t widest = R * (size_t)d.D > (size_t)d.N * d.N ? R * (size_t)d.D : (size_t)d.N * d.N;
+  const size_t fma = widest * (size_t)backward_token_chunks(d, nullptr);
+  const size_t tc = (size_t)backward_token_segments(d, nullptr) * 128 * (size_t)d.D;
+  return fma > tc ? fma : tc;
+}
+
 // Chunks of the reductions over tokens: enough of them that, with D / 512 column blocks each, about 900 CTAs are
 // in the grid (two rounds of three CTAs per SM), but no chunk shorter than 64 tokens.
 int backward_token_chunks(const Dims& d, int* chunk_tokens) {
@@ -535,6 +555,65 @@ int backward_token_chunks(const Dims& d, int* chunk_tokens) {
 }
 
 namespace {
+
+// A float factor [T, M] (M <= 64) as two bf16 terms per value: dst[t, m] = hi, dst[t, 64 + m] = lo, v = hi + lo up to
+// 2^-17 relative; unused columns are zero.
+__global__ void __launch_bounds__(256) split_bf16_kernel(const float* __restrict__ src, long long rs, int M, int T,
+                                                         __nv_bfloat16* __restrict__ dst) {
+  const long long i = (long long)blockIdx.x * 256 + threadIdx.x;
+  const long long t = i >> 6;
+  const int m = (int)(i & 63);
+  if (t >= T) return;
+  float hi = 0.f, lo = 0.f;
+  if (m < M) {
+    const float v = src[t * rs + m];
+    hi = __bfloat162float(__float2bfloat16_rn(v));
+    lo = v - hi;
+  }
+  dst[t * 128 + m] = __float2bfloat16_rn(hi);
+  dst[t * 128 + 64 + m] = __float2bfloat16_rn(lo);
+}
+
+__global__ void token_segments_kernel(int32_t* __restrict__ segs, int T, int n_seg, int per) {
+  const int i = threadIdx.x;
+  if (i <= n_seg) segs[i] = min(T, i * per);
+}
+
+// out[m, n] = sum over segments (in order) of part[seg, m, n] + part[seg, 64 + m, n] for m < M, the first rows_a rows
+// to out_a and the rest to out_b
+__global__ void __launch_bounds__(256)
+sum_split_parts_kernel(const float* __restrict__ part, float* __restrict__ out_a, int rows_a, float* __restrict__ out_b,
+                       int M, int Nout, int n_seg) {
+  const long long i = (long long)blockIdx.x * 256 + threadIdx.x;
+  if (i >= (long long)M * Nout) return;
+  const int m = (int)(i / Nout), n = (int)(i % Nout);
+  float s = 0.f;
+  for (int z = 0; z < n_seg; ++z) {
+    const float* p = part + ((size_t)z * 128 + m) * Nout + n;
+    s += p[0] + p[(size_t)64 * Nout];
+  }
+  if (m < rows_a) out_a[(size_t)m * Nout + n] = s;
+  else out_b[(size_t)(m - rows_a) * Nout + n] = s;
+}
+
+// The same reduction as token_outer on the tensor cores (bf16 activations, M <= 64, D wide enough to matter);
+// cudaErrorNotSupported when it does not apply.
+cudaError_t token_outer_tc(const Dims& d, const float* A, long long a_rs, int M, const void* B, const BackwardScratch& b,
+                           float* out_a, int rows_a, float* out_b, cudaStream_t st) {
+  if (d.dtype != MOEPP_BF16 || M > 64 || d.D < 256 || d.T < 1024) return cudaErrorNotSupported;
+  int per;
+  const int n_seg = backward_token_segments(d, &per);
+  split_bf16_kernel<<<(unsigned)(((long long)d.T * 64 + 255) / 256), 256, 0, st>>>(
+      A, a_rs, M, d.T, static_cast<__nv_bfloat16*>(b.split));
+  cudaError_t err = cudaGetLastError();
+  if (err != cudaSuccess) return err;
+  token_segments_kernel<<<1, 128, 0, st>>>(b.segs, d.T, n_seg, per);
+  if ((err = cudaGetLastError()) != cudaSuccess) return err;
+  if ((err = launch_token_outer_tc(d, b.split, B, b.part, b.segs, n_seg, st)) != cudaSuccess) return err;
+  const long long n = (long long)M * d.D;
+  sum_split_parts_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(b.part, out_a, rows_a, out_b, M, d.D, n_seg);
+  return cudaGetLastError();
+}
 
 // out_a takes the first rows_a rows of the [M, Nout] product, out_b (if any) the rest
 template <typename TB>
@@ -590,11 +669,15 @@ cudaError_t layer_backward_t(const Dims& d, const ForwardState& fs, const moepp_
   if (err != cudaSuccess) return err;
 
   // router and constant-expert weights in one product: [dG | dz]^T x, rows 0..N-1 -> dW_r, the rest -> dW_c
-  if ((err = token_outer<XT>(d, b.dGz, R, R, x, d.D, d.D, b.part, g.dW_r, d.N, g.dW_c, st)) != cudaSuccess) return err;
+  const bool fma_only = (d.flags & MOEPP_FLAG_SIMT_FFN) != 0;
+  err = fma_only ? cudaErrorNotSupported : token_outer_tc(d, b.dGz, R, R, x, b, g.dW_r, d.N, g.dW_c, st);
+  if (err == cudaErrorNotSupported) err = token_outer<XT>(d, b.dGz, R, R, x, d.D, d.D, b.part, g.dW_r, d.N, g.dW_c, st);
+  if (err != cudaSuccess) return err;
   if (d.n_const > 0) {
-    if ((err = token_outer<XT>(d, b.cvq, d.n_const, d.n_const, dy, d.D, d.D, b.part, g.dv, d.n_const, nullptr, st)) !=
-        cudaSuccess)
-      return err;
+    err = fma_only ? cudaErrorNotSupported : token_outer_tc(d, b.cvq, d.n_const, d.n_const, dy, b, g.dv, d.n_const, nullptr, st);
+    if (err == cudaErrorNotSupported)
+      err = token_outer<XT>(d, b.cvq, d.n_const, d.n_const, dy, d.D, d.D, b.part, g.dv, d.n_const, nullptr, st);
+    if (err != cudaSuccess) return err;
   }
   if (w.W_g != nullptr && g.dW_g != nullptr) {
     if ((err = token_outer<float>(d, b.dGz, R, d.N, prev, d.N, d.N, b.part, g.dW_g, d.N, nullptr, st)) != cudaSuccess)

@@ -383,6 +383,25 @@ cudaError_t run(int sms, const CUtensorMap& a0, const CUtensorMap& a1, const CUt
 
 }  // namespace
 
+// The WGRAD mode with token segments in the place of expert segments: sum over tokens of P[t, :]^T Q[t, :].
+cudaError_t launch_token_outer_tc(const Dims& d, const void* P, const void* Q, float* part, const int32_t* segs,
+                                  int n_seg, cudaStream_t st) {
+  int dev = 0, sms = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return err;
+  err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (err != cudaSuccess) return err;
+  int32_t* err_word = device_error_word();
+  if (err_word == nullptr || n_seg < 1 || n_seg > kMaxExperts) return cudaErrorNotSupported;
+  CUtensorMap mP, mQ;
+  if (!make_bf16_tile_map(&mP, P, (uint64_t)d.T, 128, 64) || !make_bf16_tile_map(&mQ, Q, (uint64_t)d.T, (uint64_t)d.D, 64))
+    return cudaErrorNotSupported;
+  Args a{};
+  a.offsets = segs; a.n_ffn = n_seg; a.err_word = err_word;
+  a.C = part; a.Mout = 128; a.Nout = d.D; a.Kd = 0;
+  return run<WGRAD>(sms, mP, mP, mQ, mQ, a, st);
+}
+
 // bf16 FFN backward on the tensor cores.  cudaErrorNotSupported when it does not apply (storage type, segments
 // that are not whole 64-row k tiles, shapes the tensor maps cannot describe): the caller then uses the FMA path.
 cudaError_t launch_ffn_backward_tc(const Dims& d, const void* x_perm, const int32_t* offsets, const void* W_gate,

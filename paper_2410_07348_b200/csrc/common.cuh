@@ -94,8 +94,20 @@ struct BackwardScratch {
   float* dGz;                   // [T, R], R = N + 2 n_const: dL/dlogits, then dL/d(mixing logits)
   float* cx;                    // [T]
   float* cvq;                   // [T, n_const]
-  float* part;                  // [chunks, max(R D, N N)] partial sums of the reductions over tokens
+  float* part;                  // partial sums of the reductions over tokens (see backward_part_floats)
+  void* split;                  // [T, 128] bf16: a small float factor as hi (columns 0..63) + lo (64..127) terms
+  int32_t* segs;                // [65] token segments of the tensor-core reduction
 };
+
+// Token segments of the tensor-core reductions (whole 64-token tiles each, at most 64 segments).
+int backward_token_segments(const Dims& d, int* tokens_per_segment);
+size_t backward_part_floats(const Dims& d);
+
+// part[seg, m, n] = sum over the tokens t of segment seg of P[t, m] Q[t, n] on the tensor cores:
+// P [T, 128] bf16 (hi | lo columns), Q [T, D] bf16, part [n_seg, 128, D] float.  cudaErrorNotSupported if the
+// tensor maps cannot be encoded.
+cudaError_t launch_token_outer_tc(const Dims& d, const void* P, const void* Q, float* part, const int32_t* segs,
+                                  int n_seg, cudaStream_t st);
 
 int backward_token_chunks(const Dims& d, int* chunk_tokens);
 
