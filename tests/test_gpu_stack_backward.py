@@ -74,20 +74,21 @@ def _layer_chain(spec, wds, cfg, x, dy, dlogits_last):
     return xs, lgs, idxs, grads
 
 
-def test_stack_backward_f32_against_oracle_chain_with_balance_loss(oracle64):
+@pytest.mark.parametrize("gamma", [0.0, 0.9])
+def test_stack_backward_f32_against_oracle_chain_with_balance_loss(oracle64, gamma):
     spec = W.LayerSpec(T=260, D=72, F=120, n_ffn=4, n_zero=1, n_copy=1, n_const=2, top_k=2, dtype="f32")
     layers = W.make_stack(spec, 3)
     for lt in layers:  # larger weights than the benchmark recipe, so that the gradients are not tiny
         lt.W_r, lt.W_gate, lt.W_up, lt.W_down = lt.W_r * 4, lt.W_gate * 3, lt.W_up * 3, lt.W_down * 3
     tau, beta = 0.75, 0.05
-    cfg = B.config_from_spec(spec, add_residual=1, tau=tau)
+    cfg = B.config_from_spec(spec, add_residual=1, tau=tau, capacity_factor=gamma)  # gamma > 0: Eq. 8 drops slots
     gen = torch.Generator().manual_seed(31)
     dy = torch.randn(spec.T, spec.D, generator=gen)
     dl_last = 0.1 * torch.randn(spec.T, spec.N, generator=gen)
     wds, x, y, lg, grads, losses = _stack_run(spec, layers, cfg, dy.cuda(), dl_last.cuda(), beta)
     _, _, idxs, _ = _layer_chain(spec, wds, cfg, x, dy.cuda(), dl_last.cuda())
 
-    s = shape_of(spec, add_residual=1, tau=tau)
+    s = shape_of(spec, add_residual=1, tau=tau, capacity_factor=gamma)
     ois = [oracle_inputs(lt) for lt in layers]
     fw, xin, prev = [], ois[0]["x"], None
     for j, o in enumerate(ois):
