@@ -148,56 +148,63 @@ route_tc_kernel(const __grid_constant__ CUtensorMap tmX, Dims dm, const float* _
     if (bias != nullptr)
       for (int i = tid_e; i < N; i += 128) s_bias[i] = bias[i];
 
-    // Each thread owns CH 16-byte chunks (8 consecutive k of one stacked row) of every 64-wide slice.  The
-    // float weights of the next slice are fetched right after this slice has been handed over, so their
-    // L2 latency is hidden behind the wait for the next free stage.
+    // Each thread owns CH 16-byte chunks (8 consecutive k of one stacked row) of every 64-wide slice.  The float
+    // weights are fetched two slices ahead of their use, so that one L2 round trip is spread over two k steps
+    // (with one slice of lookahead the loop ran at one L2 latency per step, twice the time x needs from HBM).
     constexpr int CH = RP * 8 / 128;
-    float wv[CH][8];
-    auto fetch = [&](int kb) {
+    constexpr int PF = 2;
+    float wv[PF][CH][8];
+    auto fetch = [&](int kb, float (&w)[CH][8]) {
 #pragma unroll
       for (int j = 0; j < CH; ++j) {
         const int c = tid_e + j * 128, n = c >> 3, k0 = kb * kBK + (c & 7) * 8;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) wv[j][i] = 0.f;
+        for (int i = 0; i < 8; ++i) w[j][i] = 0.f;
         if (kb < KB && n < R && k0 < D) {
           const float* src = ((n < N) ? (W_r + (size_t)n * D) : (W_c + (size_t)(n - N) * D)) + k0;
           const float4 a = __ldg(reinterpret_cast<const float4*>(src));
           const float4 b = __ldg(reinterpret_cast<const float4*>(src + 4));
-          wv[j][0] = a.x; wv[j][1] = a.y; wv[j][2] = a.z; wv[j][3] = a.w;
-          wv[j][4] = b.x; wv[j][5] = b.y; wv[j][6] = b.z; wv[j][7] = b.w;
+          w[j][0] = a.x; w[j][1] = a.y; w[j][2] = a.z; w[j][3] = a.w;
+          w[j][4] = b.x; w[j][5] = b.y; w[j][6] = b.z; w[j][7] = b.w;
         }
       }
     };
-    fetch(0);
+#pragma unroll
+    for (int u = 0; u < PF; ++u) fetch(u, wv[u]);
     bool ok = true;
-    for (int kb = 0; kb < KB && ok; ++kb) {
-      const uint32_t s = kb % kStagesR, ph = (kb / kStagesR) & 1u;
-      if (!mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u, &abort_flag, 13, err_word)) { ok = false; break; }
-      uint8_t* bbase = ring_ptr + s * L::kStage + kABytesR;
+    for (int kb0 = 0; kb0 < KB && ok; kb0 += PF) {
 #pragma unroll
-      for (int j = 0; j < CH; ++j) {
-        const int c = tid_e + j * 128, n = c >> 3, kc = c & 7;
-        float hi[8], mid[8], lo[8];
+      for (int u = 0; u < PF; ++u) {
+        const int kb = kb0 + u;
+        if (kb >= KB || !ok) break;
+        const uint32_t s = kb % kStagesR, ph = (kb / kStagesR) & 1u;
+        if (!mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u, &abort_flag, 13, err_word)) { ok = false; break; }
+        uint8_t* bbase = ring_ptr + s * L::kStage + kABytesR;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          hi[i] = __bfloat162float(__float2bfloat16_rn(wv[j][i]));
-          const float r1 = wv[j][i] - hi[i];  // exact
-          mid[i] = __bfloat162float(__float2bfloat16_rn(r1));
-          lo[i] = r1 - mid[i];                // exact; rounded to bf16 when packed
+        for (int j = 0; j < CH; ++j) {
+          const int c = tid_e + j * 128, n = c >> 3, kc = c & 7;
+          float hi[8], mid[8], lo[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            hi[i] = __bfloat162float(__float2bfloat16_rn(wv[u][j][i]));
+            const float r1 = wv[u][j][i] - hi[i];  // exact
+            mid[i] = __bfloat162float(__float2bfloat16_rn(r1));
+            lo[i] = r1 - mid[i];                   // exact; rounded to bf16 when packed
+          }
+          const int off = (n >> 3) * 1024 + (n & 7) * 128 + ((kc ^ (n & 7)) << 4);
+          *reinterpret_cast<uint4*>(bbase + off) = make_uint4(pack_bf16(hi[0], hi[1]), pack_bf16(hi[2], hi[3]),
+                                                              pack_bf16(hi[4], hi[5]), pack_bf16(hi[6], hi[7]));
+          *reinterpret_cast<uint4*>(bbase + L::kBSub + off) =
+              make_uint4(pack_bf16(mid[0], mid[1]), pack_bf16(mid[2], mid[3]), pack_bf16(mid[4], mid[5]),
+                         pack_bf16(mid[6], mid[7]));
+          *reinterpret_cast<uint4*>(bbase + 2 * L::kBSub + off) =
+              make_uint4(pack_bf16(lo[0], lo[1]), pack_bf16(lo[2], lo[3]), pack_bf16(lo[4], lo[5]),
+                         pack_bf16(lo[6], lo[7]));
         }
-        const int off = (n >> 3) * 1024 + (n & 7) * 128 + ((kc ^ (n & 7)) << 4);
-        *reinterpret_cast<uint4*>(bbase + off) = make_uint4(pack_bf16(hi[0], hi[1]), pack_bf16(hi[2], hi[3]),
-                                                            pack_bf16(hi[4], hi[5]), pack_bf16(hi[6], hi[7]));
-        *reinterpret_cast<uint4*>(bbase + L::kBSub + off) =
-            make_uint4(pack_bf16(mid[0], mid[1]), pack_bf16(mid[2], mid[3]), pack_bf16(mid[4], mid[5]),
-                       pack_bf16(mid[6], mid[7]));
-        *reinterpret_cast<uint4*>(bbase + 2 * L::kBSub + off) =
-            make_uint4(pack_bf16(lo[0], lo[1]), pack_bf16(lo[2], lo[3]), pack_bf16(lo[4], lo[5]),
-                       pack_bf16(lo[6], lo[7]));
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the MMA
+        mbar_arrive(smem_u32(&bar_full[s]));
+        fetch(kb + PF, wv[u]);
       }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the MMA
-      mbar_arrive(smem_u32(&bar_full[s]));
-      fetch(kb + 1);
     }
     if (ok) ok = mbar_wait(smem_u32(&bar_tmem_full), 0, &abort_flag, 14, err_word);
     named_barrier_128();
