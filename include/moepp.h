@@ -211,8 +211,8 @@ moepp_status moepp_balance_backward(const moepp_config* cfg, const float* logits
  * logits_out (may be NULL) the last layer's logits.  Workspace: moepp_stack_workspace_bytes().
  * The _host variant takes host pointers for x, prev_logits, y and logits_out (pinned memory for
  * asynchronous copies): x goes to the device once, y comes back once, the layers in between stay on
- * the device.  For T >= 4096 (and no capacity limit) the tokens are cut into 2 or 4 chunks that are
- * pipelined: one chunk computes on `stream` while the next is copied in and the previous is copied out
+ * the device.  For T >= 4096 (and no capacity limit) the tokens are cut into 2 or 4 chunks (equal ones, or
+ * 1/8, 3/8, 3/8, 1/8 when the stack's arithmetic outlasts the copies) that are pipelined: one chunk computes on `stream` while the next is copied in and the previous is copied out
  * on two internal streams; these streams and the events that order them are created and released
  * inside the call (no device memory is allocated), `stream` is made to wait for the last copy, and the
  * results are the same bits as without chunking.  Workspace: moepp_stack_workspace_bytes_host().

@@ -387,18 +387,41 @@ moepp_status moepp_stack_forward(const moepp_config* cfg, const moepp_weights* l
 namespace {
 
 struct HostChunks {
-  int n;        // number of chunks
-  int tokens;   // tokens per chunk (a multiple of 128; the last chunk takes the rest)
+  int n;           // number of chunks
+  int begin[4];    // first token of each chunk
+  int tokens[4];   // tokens of each chunk (multiples of 128; the last chunk takes the rest)
 };
 
-HostChunks host_chunks(const Dims& d) {
-  HostChunks h{1, d.T};
-  if (d.cap_on) return h;  // Eq. 8 shares one capacity among all tokens: keep the batch whole
-  const int n = d.T >= 16384 ? 4 : (d.T >= 4096 ? 2 : 1);
-  if (n > 1) {
-    h.n = n;
-    h.tokens = ((d.T + n - 1) / n + 127) / 128 * 128;
-    h.n = (d.T + h.tokens - 1) / h.tokens;
+// Large batches are cut into 4 chunks (2 from 4096 tokens on).  Where the stack's arithmetic outlasts the copies
+// (about n_layers * F * K >= 16384 at PCIe 5 and bf16 tensor speed) the cut is 1/8, 3/8, 3/8, 1/8: a short copy-in
+// before compute starts, a short copy-out tail, and middle chunks whose GEMMs run at nearly the full batch's
+// efficiency.  Otherwise the copies are the bound and equal chunks keep both copy directions busy longest.
+HostChunks host_chunks(const Dims& d, int n_layers) {
+  HostChunks h{};
+  h.n = 1; h.begin[0] = 0; h.tokens[0] = d.T;
+  if (d.cap_on || d.T < 4096) return h;  // Eq. 8 shares one capacity among all tokens: keep the batch whole
+  auto up128 = [](long long v) { return (int)((v + 127) / 128 * 128); };
+  const bool compute_bound = (long long)n_layers * d.F * d.K >= 16384;
+  int want[4], n;
+  if (d.T >= 16384) {
+    n = 4;
+    if (compute_bound) {
+      want[0] = up128(d.T / 8); want[1] = up128(3LL * d.T / 8); want[2] = want[1];
+    } else {
+      want[0] = want[1] = want[2] = up128((d.T + 3) / 4);
+    }
+    want[3] = d.T;
+  } else {
+    n = 2;
+    want[0] = up128(d.T / 2); want[1] = d.T;
+  }
+  int at = 0;
+  h.n = 0;
+  for (int i = 0; i < n && at < d.T; ++i) {
+    const int tok = (i + 1 < n && at + want[i] < d.T) ? want[i] : d.T - at;
+    h.begin[h.n] = at; h.tokens[h.n] = tok;
+    at += tok;
+    ++h.n;
   }
   return h;
 }
@@ -427,12 +450,9 @@ moepp_status moepp_stack_workspace_bytes_host(const moepp_config* cfg, int32_t n
   const moepp_status s = make_dims(cfg, &d);
   if (s != MOEPP_OK) return s;
   if (bytes == nullptr || n_layers < 1) return MOEPP_ERR_INVALID_ARG;
-  const HostChunks h = host_chunks(d);
+  const HostChunks h = host_chunks(d, n_layers);
   size_t total = 0;
-  for (int i = 0; i < h.n; ++i) {
-    const int tok = (i + 1 < h.n) ? h.tokens : d.T - i * h.tokens;
-    total += chunk_ws_bytes(chunk_dims(d, tok, h.n > 1));
-  }
+  for (int i = 0; i < h.n; ++i) total += chunk_ws_bytes(chunk_dims(d, h.tokens[i], h.n > 1));
   *bytes = total;
   return MOEPP_OK;
 }
@@ -455,7 +475,7 @@ moepp_status moepp_stack_forward_host(const moepp_config* cfg, const moepp_weigh
   if (d.T > 0 && layers[0].W_g != nullptr && prev_logits_host == nullptr) return MOEPP_ERR_INVALID_ARG;
   if (d.T == 0) return MOEPP_OK;
 
-  const HostChunks h = host_chunks(d);
+  const HostChunks h = host_chunks(d, n_layers);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const size_t es = elem_size(d.dtype);
   constexpr int kMaxChunks = 8;
@@ -483,8 +503,7 @@ moepp_status moepp_stack_forward_host(const moepp_config* cfg, const moepp_weigh
 
   char* ws = static_cast<char*>(workspace);
   for (int i = 0; i < h.n && result == MOEPP_OK; ++i) {
-    const int t_begin = i * h.tokens;
-    const int tok = (i + 1 < h.n) ? h.tokens : d.T - t_begin;
+    const int t_begin = h.begin[i], tok = h.tokens[i];
     const Dims c = chunk_dims(d, tok, h.n > 1);
     size_t act, lg;
     const size_t extra = stack_extra_bytes(c, &act, &lg);
