@@ -66,6 +66,10 @@ typedef enum { MOEPP_F32 = 0, MOEPP_BF16 = 1 } moepp_dtype;
 #define MOEPP_FLAG_SAVE_PREACT 16 /* moepp_layer_forward: also keep the SwiGLU pre-activations (gate and up, [M_cap, F]
                                      each) in the workspace, which grows accordingly; moepp_layer_backward then skips
                                      their recomputation.  Not with MOEPP_FLAG_FFN_SINGLE_CTA / MOEPP_FLAG_FUSED_GATHER. */
+#define MOEPP_FLAG_ACCUM_GRADS 32 /* moepp_layer_backward / moepp_stack_backward: ADD the weight gradients (dW_r, dW_g,
+                                     dbias, dW_c, dv, dW_gate, dW_up, dW_down) to what the buffers hold instead of
+                                     overwriting them (gradient accumulation over micro-batches); dx and dprev are
+                                     always overwritten */
 
 typedef struct {
   int32_t T, D, F;
@@ -232,7 +236,7 @@ moepp_status moepp_stack_forward_host(const moepp_config* cfg, const moepp_weigh
  * prints no formulas for it; these are the derivatives of the forward pass above.
  *
  * Every pointer of moepp_grads is device memory the caller owns; every gradient is OVERWRITTEN
- * (not accumulated).  Weight gradients are float whatever cfg->dtype is; dx has cfg->dtype.
+ * (with MOEPP_FLAG_ACCUM_GRADS the weight gradients are added to instead).  Weight gradients are float whatever cfg->dtype is; dx has cfg->dtype.
  */
 typedef struct {
   void* dx;       /* [T, D]  dL/dx, cfg->dtype */

@@ -17,7 +17,7 @@ _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libmoepp.s
 _lib = None
 
 MOEPP_F32, MOEPP_BF16 = 0, 1
-FLAG_LOGITS_GIVEN, FLAG_SIMT_FFN, FLAG_FFN_SINGLE_CTA, FLAG_FUSED_GATHER, FLAG_SAVE_PREACT = 1, 2, 4, 8, 16
+FLAG_LOGITS_GIVEN, FLAG_SIMT_FFN, FLAG_FFN_SINGLE_CTA, FLAG_FUSED_GATHER, FLAG_SAVE_PREACT, FLAG_ACCUM_GRADS = 1, 2, 4, 8, 16, 32
 STATUS = {0: "MOEPP_OK", 1: "MOEPP_ERR_INVALID_ARG", 2: "MOEPP_ERR_UNSUPPORTED", 3: "MOEPP_ERR_ALIGN",
           4: "MOEPP_ERR_WORKSPACE", 5: "MOEPP_ERR_CUDA", 6: "MOEPP_ERR_TIMEOUT"}
 

@@ -246,18 +246,19 @@ token_outer_kernel(const float* __restrict__ A, const TB* __restrict__ B, float*
 
 // sum over z (in order) of part[z, i], written to out_a[i] for i < n_a and to out_b[i - n_a] after that
 __global__ void __launch_bounds__(256) sum_parts_kernel(const float* __restrict__ part, float* __restrict__ out_a,
-                                                        long long n_a, float* __restrict__ out_b, long long n, int Z) {
+                                                        long long n_a, float* __restrict__ out_b, long long n, int Z,
+                                                        int accumulate) {
   const long long i = (long long)blockIdx.x * 256 + threadIdx.x;
   if (i >= n) return;
   float s = 0.f;
   for (int z = 0; z < Z; ++z) s += part[(size_t)z * n + i];
-  if (i < n_a) out_a[i] = s;
-  else out_b[i - n_a] = s;
+  float* dst = i < n_a ? out_a + i : out_b + (i - n_a);
+  *dst = accumulate ? *dst + s : s;
 }
 
 // out[i] = sum over tokens of A[t, i]; one block per column, fixed order of the partial sums
 __global__ void __launch_bounds__(256) column_sum_kernel(const float* __restrict__ A, float* __restrict__ out, int T,
-                                                         long long a_rs) {
+                                                         long long a_rs, int accumulate) {
   __shared__ float s[256];
   float acc = 0.f;
   for (int t = threadIdx.x; t < T; t += 256) acc += A[(size_t)t * a_rs + blockIdx.x];
@@ -267,7 +268,7 @@ __global__ void __launch_bounds__(256) column_sum_kernel(const float* __restrict
     if ((int)threadIdx.x < o) s[threadIdx.x] += s[threadIdx.x + o];
     __syncthreads();
   }
-  if (threadIdx.x == 0) out[blockIdx.x] = s[0];
+  if (threadIdx.x == 0) out[blockIdx.x] = accumulate ? out[blockIdx.x] + s[0] : s[0];
 }
 
 constexpr int kDxTokens = 4;   // tokens per warp in dx_assemble
@@ -583,7 +584,7 @@ __global__ void token_segments_kernel(int32_t* __restrict__ segs, int T, int n_s
 // to out_a and the rest to out_b
 __global__ void __launch_bounds__(256)
 sum_split_parts_kernel(const float* __restrict__ part, float* __restrict__ out_a, int rows_a, float* __restrict__ out_b,
-                       int M, int Nout, int n_seg) {
+                       int M, int Nout, int n_seg, int accumulate) {
   const long long i = (long long)blockIdx.x * 256 + threadIdx.x;
   if (i >= (long long)M * Nout) return;
   const int m = (int)(i / Nout), n = (int)(i % Nout);
@@ -592,8 +593,8 @@ sum_split_parts_kernel(const float* __restrict__ part, float* __restrict__ out_a
     const float* p = part + ((size_t)z * 128 + m) * Nout + n;
     s += p[0] + p[(size_t)64 * Nout];
   }
-  if (m < rows_a) out_a[(size_t)m * Nout + n] = s;
-  else out_b[(size_t)(m - rows_a) * Nout + n] = s;
+  float* dst = m < rows_a ? out_a + (size_t)m * Nout + n : out_b + (size_t)(m - rows_a) * Nout + n;
+  *dst = accumulate ? *dst + s : s;
 }
 
 // The same reduction as token_outer on the tensor cores (bf16 activations, M <= 64, D wide enough to matter);
@@ -611,7 +612,8 @@ cudaError_t token_outer_tc(const Dims& d, const float* A, long long a_rs, int M,
   if ((err = cudaGetLastError()) != cudaSuccess) return err;
   if ((err = launch_token_outer_tc(d, b.split, B, b.part, b.segs, n_seg, st)) != cudaSuccess) return err;
   const long long n = (long long)M * d.D;
-  sum_split_parts_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(b.part, out_a, rows_a, out_b, M, d.D, n_seg);
+  sum_split_parts_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(b.part, out_a, rows_a, out_b, M, d.D, n_seg,
+                                                                      (d.flags & MOEPP_FLAG_ACCUM_GRADS) ? 1 : 0);
   return cudaGetLastError();
 }
 
@@ -634,7 +636,8 @@ cudaError_t token_outer(const Dims& d, const float* A, long long a_rs, int M, co
   cudaError_t err = cudaGetLastError();
   if (err != cudaSuccess) return err;
   const long long n = (long long)M * Nout;
-  sum_parts_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(part, out_a, (long long)rows_a * Nout, out_b, n, Z);
+  sum_parts_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(part, out_a, (long long)rows_a * Nout, out_b, n, Z,
+                                                                (d.flags & MOEPP_FLAG_ACCUM_GRADS) ? 1 : 0);
   return cudaGetLastError();
 }
 
@@ -684,7 +687,7 @@ cudaError_t layer_backward_t(const Dims& d, const ForwardState& fs, const moepp_
       return err;
   }
   if (g.dbias != nullptr) {
-    column_sum_kernel<<<(unsigned)d.N, 256, 0, st>>>(b.dGz, g.dbias, d.T, R);
+    column_sum_kernel<<<(unsigned)d.N, 256, 0, st>>>(b.dGz, g.dbias, d.T, R, (d.flags & MOEPP_FLAG_ACCUM_GRADS) ? 1 : 0);
     if ((err = cudaGetLastError()) != cudaSuccess) return err;
   }
   const int dx_tokens = kWarpsPerBlock * kDxTokens * kDxGroups;
@@ -706,6 +709,7 @@ cudaError_t layer_backward_t(const Dims& d, const ForwardState& fs, const moepp_
 cudaError_t launch_layer_backward(const Dims& d, const ForwardState& fs, const moepp_weights& w, const void* x,
                                   const float* prev, const void* dy, const float* dlogits_next,
                                   const BackwardScratch& b, const moepp_grads& g, cudaStream_t st) {
+  if (d.T == 0 && (d.flags & MOEPP_FLAG_ACCUM_GRADS)) return cudaSuccess;  // no tokens, nothing to add
   if (d.T == 0) {  // no tokens: every weight gradient is zero
     const int R2 = 2 * d.n_const;
     cudaError_t err;

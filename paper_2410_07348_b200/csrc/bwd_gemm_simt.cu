@@ -98,7 +98,8 @@ __global__ void __launch_bounds__(256) bwd_rows_kernel(RowsArgs a) {
 template <typename T>
 __global__ void __launch_bounds__(256)
 bwd_wgrad_kernel(const T* __restrict__ A, const T* __restrict__ B, float* __restrict__ C,
-                 const int32_t* __restrict__ offsets, int Mout, int Nout, long long a_rs, long long b_rs) {
+                 const int32_t* __restrict__ offsets, int Mout, int Nout, long long a_rs, long long b_rs,
+                 int accumulate) {
   __shared__ float As[TK][TM + 4], Bs[TK][TN + 4];
   const int e = blockIdx.z, m0 = blockIdx.x * TM, n0 = blockIdx.y * TN;
   const int r_begin = offsets[e], r_end = offsets[e + 1];
@@ -131,7 +132,10 @@ bwd_wgrad_kernel(const T* __restrict__ A, const T* __restrict__ B, float* __rest
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const int m = m0 + ty * 4 + i, n = n0 + tx * 4 + j;
-      if (m < Mout && n < Nout) C[((size_t)e * Mout + m) * Nout + n] = acc[i][j];
+      if (m < Mout && n < Nout) {
+        float* dst = C + ((size_t)e * Mout + m) * Nout + n;
+        *dst = accumulate ? *dst + acc[i][j] : acc[i][j];
+      }
     }
 }
 
@@ -153,6 +157,7 @@ cudaError_t ffn_backward_t(const Dims& d, const void* x_perm, const int32_t* off
                            void* up_buf, void* dx_perm, float* dW_gate, float* dW_up, float* dW_down,
                            cudaStream_t st, const void* gate_in, const void* up_in) {
   const long long D = d.D, F = d.F;
+  const int accum = (d.flags & MOEPP_FLAG_ACCUM_GRADS) ? 1 : 0;
   cudaError_t err;
   if (gate_in == nullptr) {
     // 1-2. SwiGLU pre-activations again: gate = Xp W_gate^T, up = Xp W_up^T
@@ -169,7 +174,7 @@ cudaError_t ffn_backward_t(const Dims& d, const void* x_perm, const int32_t* off
   // 3. dW_down[e] = dYp_e^T H_e
   dim3 gdn((unsigned)((d.D + TM - 1) / TM), (unsigned)((d.F + TN - 1) / TN), (unsigned)d.n_ffn);
   bwd_wgrad_kernel<T><<<gdn, 256, 0, st>>>(static_cast<const T*>(dy_perm), static_cast<const T*>(h), dW_down, offsets,
-                                           d.D, d.F, D, F);
+                                           d.D, d.F, D, F, accum);
   if ((err = cudaGetLastError()) != cudaSuccess) return err;
   // 4. dH = dYp W_down, turned in place into dGate, dUp
   RowsArgs b{};
@@ -180,10 +185,10 @@ cudaError_t ffn_backward_t(const Dims& d, const void* x_perm, const int32_t* off
   // 5. dW_gate[e] = dGate_e^T Xp_e, dW_up[e] = dUp_e^T Xp_e
   dim3 gup((unsigned)((d.F + TM - 1) / TM), (unsigned)((d.D + TN - 1) / TN), (unsigned)d.n_ffn);
   bwd_wgrad_kernel<T><<<gup, 256, 0, st>>>(static_cast<const T*>(gate_buf), static_cast<const T*>(x_perm), dW_gate,
-                                           offsets, d.F, d.D, F, D);
+                                           offsets, d.F, d.D, F, D, accum);
   if ((err = cudaGetLastError()) != cudaSuccess) return err;
   bwd_wgrad_kernel<T><<<gup, 256, 0, st>>>(static_cast<const T*>(up_buf), static_cast<const T*>(x_perm), dW_up, offsets,
-                                           d.F, d.D, F, D);
+                                           d.F, d.D, F, D, accum);
   if ((err = cudaGetLastError()) != cudaSuccess) return err;
   // 6. dXp = dGate W_gate + dUp W_up
   RowsArgs c{};
@@ -204,6 +209,7 @@ cudaError_t launch_ffn_backward_simt(const Dims& d, const void* x_perm, const in
   if (d.n_ffn == 0) return cudaSuccess;
   const size_t wbytes = sizeof(float) * (size_t)d.n_ffn * d.D * d.F;
   cudaError_t err;  // experts without rows still get a defined (zero) gradient
+  if ((d.T == 0 || d.M_cap == 0) && (d.flags & MOEPP_FLAG_ACCUM_GRADS)) return cudaSuccess;  // nothing to add
   if (d.T == 0 || d.M_cap == 0) {
     if ((err = cudaMemsetAsync(dW_gate, 0, wbytes, st)) != cudaSuccess) return err;
     if ((err = cudaMemsetAsync(dW_up, 0, wbytes, st)) != cudaSuccess) return err;

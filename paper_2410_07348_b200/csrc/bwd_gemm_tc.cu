@@ -58,6 +58,7 @@ struct Args {
   const __nv_bfloat16 *gate_in, *up_in;  // DH: pre-activations in (may be the same buffers)
   const int32_t* offsets;
   int n_ffn, Mout, Nout, Kd;
+  int accumulate;          // WGRAD: add to C instead of overwriting it
   int32_t* err_word;
 };
 
@@ -245,11 +246,17 @@ bwd_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant_
           if (row_ok) {
 #pragma unroll
             for (int v = 0; v < 4; ++v)
-              if (ti.n0 + c + 4 * v + 4 <= a.Nout)
-                *reinterpret_cast<float4*>(crow + c + 4 * v) =
-                    empty ? make_float4(0.f, 0.f, 0.f, 0.f)
-                          : make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
-                                        __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
+              if (ti.n0 + c + 4 * v + 4 <= a.Nout) {
+                float4 o = empty ? make_float4(0.f, 0.f, 0.f, 0.f)
+                                 : make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                               __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
+                float4* dst = reinterpret_cast<float4*>(crow + c + 4 * v);
+                if (a.accumulate) {
+                  const float4 old = *dst;
+                  o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+                }
+                *dst = o;
+              }
           }
         }
       } else {
@@ -444,6 +451,7 @@ cudaError_t launch_ffn_backward_tc(const Dims& d, const void* x_perm, const int3
   Args a{};
   a.offsets = offsets; a.n_ffn = d.n_ffn; a.err_word = err_word;
   // 2. dW_down[e] = dYp_e^T H_e
+  a.accumulate = (d.flags & MOEPP_FLAG_ACCUM_GRADS) ? 1 : 0;
   a.C = dW_down; a.Mout = d.D; a.Nout = d.F; a.Kd = 0;
   if ((err = run<WGRAD>(sms, mDyMN, mDyMN, mHMN, mHMN, a, st)) != cudaSuccess) return err;
   // 3. dH = dYp W_down -> dGate, dUp in place

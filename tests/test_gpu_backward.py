@@ -251,6 +251,42 @@ def test_backward_full_size_layer_on_sampled_tokens(oracle64):
         assert err <= TOL["bf16"], (name, err)
 
 
+@pytest.mark.parametrize("dtype,row_align", [("f32", 1), ("bf16", 64), ("bf16", 8)])
+def test_backward_gradient_accumulation(dtype, row_align):
+    """MOEPP_FLAG_ACCUM_GRADS: two calls into zeroed buffers give exactly twice the weight gradients of one plain call
+    (g + g is exact in float); dx and dprev are overwritten, not added to."""
+    spec = W.LayerSpec(T=1300, D=264, F=200, n_ffn=5, n_zero=1, n_copy=1, n_const=2, top_k=2, dtype=dtype)
+    lt = W.make_layer(spec, seed=17, with_prev=True, w_std=0.05)
+    wd = B.weights_from_tensors(lt)
+    x, prev = lt.x.cuda(), lt.prev.cuda()
+    gen = torch.Generator().manual_seed(3)
+    dy = torch.randn(spec.T, spec.D, generator=gen).to(x.dtype).cuda()
+    dev = "cuda"
+    outs = []
+    for flags, calls in ((0, 1), (B.FLAG_ACCUM_GRADS, 2)):
+        cfg = B.config_from_spec(spec, row_align=row_align, flags=flags)
+        ws = torch.empty(B.moepp_workspace_bytes(cfg), dtype=torch.uint8, device=dev)
+        bws = torch.empty(B.moepp_backward_workspace_bytes(cfg), dtype=torch.uint8, device=dev)
+        y, logits = torch.empty_like(x), torch.empty(spec.T, spec.N, device=dev)
+        B.moepp_layer_forward(cfg, wd, x, prev, y, logits, ws)
+        z = lambda *shape, dt=torch.float32: torch.zeros(*shape, dtype=dt, device=dev)
+        N, D, F = spec.N, spec.D, spec.F
+        g = dict(dx=z(spec.T, D, dt=x.dtype), dprev=z(spec.T, N), dW_r=z(N, D), dW_g=z(N, N), dbias=z(N),
+                 dW_c=z(spec.n_const, 2, D), dv=z(spec.n_const, D), dW_gate=z(spec.n_ffn, F, D),
+                 dW_up=z(spec.n_ffn, F, D), dW_down=z(spec.n_ffn, D, F))
+        for _ in range(calls):
+            B.moepp_layer_backward(cfg, wd, x, prev, logits, dy, None, ws, g, bws)
+        torch.cuda.synchronize()
+        outs.append(g)
+    one, two = outs
+    for name in GRADS:
+        if name in ("dx", "dprev"):
+            assert torch.equal(one[name], two[name]), name
+        else:
+            assert torch.equal(2 * one[name], two[name]), name
+            assert one[name].abs().max() > 0, name
+
+
 def test_backward_no_tokens():
     spec = W.LayerSpec(T=0, D=64, F=96, n_ffn=2, n_zero=1, n_copy=1, n_const=1, top_k=2, dtype="f32")
     lt = W.make_layer(spec, seed=0, with_prev=True)
