@@ -87,6 +87,48 @@ def test_null_config_and_null_outputs(lib):
     assert lib.moepp_stack_forward_host(ctypes.byref(c), null, 1, *([null] * 5), ctypes.c_size_t(0), null) == 1
 
 
+def test_backward_sizing_and_argument_checks_are_host_only(lib):
+    """The backward and training-stack entry points: workspace sizes are pure host arithmetic, and bad arguments come
+    back as status codes before anything is launched."""
+    cfg = B.Config(T=512, D=256, F=512, n_ffn=8, n_zero=1, n_copy=1, n_const=2, row_align=64)
+    kept = B.Config(T=512, D=256, F=512, n_ffn=8, n_zero=1, n_copy=1, n_const=2, row_align=64, flags=B.FLAG_SAVE_PREACT)
+    bwd = B.moepp_backward_workspace_bytes(cfg)
+    rows, es = cfg.M_cap, 2
+    assert bwd % 256 == 0 and bwd >= rows * (2 * 256 + 2 * 512) * es  # dYp, dXp, gate, up
+    # keeping the pre-activations adds two [M_cap, F] buffers to the forward workspace
+    assert B.moepp_workspace_bytes(kept) - B.moepp_workspace_bytes(cfg) >= 2 * rows * 512 * es
+    one_slot = B.moepp_stack_train_workspace_bytes(cfg, 1)
+    assert B.moepp_stack_train_workspace_bytes(cfg, 3) == 3 * one_slot
+    assert one_slot > B.moepp_workspace_bytes(cfg)
+    assert B.moepp_stack_backward_workspace_bytes(cfg, 3) > bwd
+    with pytest.raises(B.MoeppError):
+        B.moepp_stack_train_workspace_bytes(cfg, 0)
+
+    c = cfg.c()
+    null, one = ctypes.c_void_p(0), ctypes.c_void_p(256)
+    sz = ctypes.c_size_t(1 << 40)
+    w = B.moepp_weights(*([256] * 8))
+    g = B.moepp_grads()
+    # no gradient set, no scratch
+    assert lib.moepp_layer_backward(ctypes.byref(c), ctypes.byref(w), one, one, null, one, null, one, sz, None, one, sz,
+                                    null) == 1
+    # a gradient set without dW_r
+    assert lib.moepp_layer_backward(ctypes.byref(c), ctypes.byref(w), one, one, null, one, null, one, sz,
+                                    ctypes.byref(g), one, sz, null) == 1
+    # workspaces too small: status 5 (workspace), checked before the gradient set is looked at
+    assert lib.moepp_layer_backward(ctypes.byref(c), ctypes.byref(w), one, one, null, one, null, one,
+                                    ctypes.c_size_t(16), ctypes.byref(g), one, ctypes.c_size_t(16), null) == \
+        lib.moepp_layer_forward(ctypes.byref(c), ctypes.byref(w), one, one, one, null, one, ctypes.c_size_t(16), null)
+    # the fused-gather forward keeps no x_perm, so it cannot be differentiated
+    fused = B.Config(T=512, D=256, F=512, n_ffn=8, flags=B.FLAG_FUSED_GATHER).c()
+    assert lib.moepp_layer_backward(ctypes.byref(fused), ctypes.byref(w), one, one, null, one, null, one, sz,
+                                    ctypes.byref(g), one, sz, null) == 1
+    assert lib.moepp_balance_backward(ctypes.byref(c), null, null, ctypes.c_float(1.0), 0, null, null) == 1
+    assert lib.moepp_stack_forward_train(ctypes.byref(c), null, 1, *([null] * 5), ctypes.c_size_t(0), null) == 1
+    assert lib.moepp_stack_backward(ctypes.byref(c), null, 1, null, null, null, null, ctypes.c_float(0.0), null, null,
+                                    ctypes.c_size_t(0), None, null, ctypes.c_size_t(0), null) == 1
+
+
 def test_missing_library_is_a_hard_error(monkeypatch):
     monkeypatch.setattr(B, "_lib", None)
     monkeypatch.setattr(B, "_LIB_PATH", "/nonexistent/libmoepp.so")
