@@ -211,6 +211,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="use only the first N layers of the workload (profiling)")
     ap.add_argument("--flags", type=int, default=0, help="MOEPP_FLAG_* bits passed in the configuration")
     ap.add_argument("--no-backward", action="store_true", help="skip the backward-pass timing of layer 1")
+    ap.add_argument("--backward-row-align", type=int, default=64, help="row_align of the backward-pass timings")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "moepp" else args.warmup
 
@@ -357,7 +358,7 @@ def main():
 
         def fwd_bwd(flags, gemm_units):
             cfg_b = B.config_from_spec(spec, add_residual=add_res, flags=flags, tau=args.tau,
-                                       capacity_factor=args.capacity_factor, row_align=64)
+                                       capacity_factor=args.capacity_factor, row_align=args.backward_row_align)
             ws_f = torch.empty(B.moepp_workspace_bytes(cfg_b), dtype=torch.uint8, device=dev)
             ws_b = torch.empty(B.moepp_backward_workspace_bytes(cfg_b), dtype=torch.uint8, device=dev)
             pair = [("forward", lambda: B.moepp_layer_forward(cfg_b, wd, x0, p1, yb, lgs[0], ws_f)),
@@ -384,15 +385,15 @@ def main():
                     "tokens_per_s_fwd_bwd": world * T / ((acc_b["forward"] + acc_b["backward"]) * 1e-3)}
 
         # dH 2, dXp 4, three weight gradients 6 (x M D F); recomputing gate and up adds 4
-        bwd = {"what": "layer 1, segments padded to 64 rows; backward = moepp_layer_backward (all gradients); "
-                       "roofline = FFN GEMM flops of the pass at the bf16 burst peak",
+        bwd = {"what": "layer 1, segments padded to %d rows; backward = moepp_layer_backward (all gradients); "
+                       "roofline = FFN GEMM flops of the pass at the bf16 burst peak" % args.backward_row_align,
                "kept_pre_activations": fwd_bwd(args.flags | B.FLAG_SAVE_PREACT, 12.0),
                "recomputed_pre_activations": fwd_bwd(args.flags, 16.0)}
         del grads
 
         # whole stack, forward (every layer keeps its state) + backward with the Eq. 7 gradient of every layer
         cfg_t = B.config_from_spec(spec, add_residual=add_res, flags=args.flags | B.FLAG_SAVE_PREACT, tau=args.tau,
-                                   capacity_factor=args.capacity_factor, row_align=64)
+                                   capacity_factor=args.capacity_factor, row_align=args.backward_row_align)
         tws = torch.empty(B.moepp_stack_train_workspace_bytes(cfg_t, L), dtype=torch.uint8, device=dev)
         sbw = torch.empty(B.moepp_stack_backward_workspace_bytes(cfg_t, L), dtype=torch.uint8, device=dev)
         glist = []

@@ -265,8 +265,9 @@ moepp_status moepp_backward_workspace_bytes(const moepp_config* cfg, size_t* byt
  * nothing, Eq. 4 passes w dy to x, Eq. 5 also feeds dv and the two mixing logits), gate backward (softmax
  * over all N, renormalisation if on), the expert FFNs (SwiGLU pre-activations recomputed from x_perm),
  * the router (dW_r, dW_g, dbias, dprev) and dx.  Slots dropped by Eq. 8 carry no gradient.
- * bf16 with row_align a multiple of 64: the FFN GEMMs run on the tensor cores, operands read in place (the
- * transposed products take their tiles MN-major); otherwise on the FMA units.  Float accumulation either way.
+ * bf16: the FFN GEMMs run on the tensor cores, operands read in place (the transposed products take their tiles
+ * MN-major); a row_align that is a multiple of 64 saves the weight-gradient kernel the clearing of one tile tail
+ * per output tile.  Float storage: FMA units.  Float accumulation either way.
  * With MOEPP_FLAG_SAVE_PREACT (set in the forward call too) the pre-activations are read from fwd_workspace
  * instead of being recomputed.
  * MOEPP_FLAG_FUSED_GATHER is refused (that forward path does not keep x_perm).

@@ -10,8 +10,8 @@
 //   DX    : dXp[r, d]  = sum_f dGate[r, f] W_gate[e][f, d] + sum_f dUp[r, f] W_up[e][f, d]
 //                                                                   A K-major, B MN-major, two k passes
 //   WGRAD : dW[e][m, n] = sum over the rows r of expert e of P[r, m] Q[r, n]   A and B MN-major, float out
-//           (the rows of an expert are the k range; every segment must be a whole number of 64-row k tiles,
-//           i.e. row_align a multiple of 64, with zero pad rows)
+//           (the rows of an expert are the k range; where a segment is not a whole number of 64-row k tiles the
+//           rows of its last tile that lie beyond it are cleared in shared memory before the MMAs)
 // Every wait is bounded: a wait that runs out raises the error word and the CTA drains and leaves.
 #include <cuda.h>
 
@@ -188,10 +188,15 @@ bwd_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant_
     }
   } else if (warp == 1) {
     // ---------------------------------- MMA issuer -----------------------------------------------
+    // Where a WGRAD k tile reaches past the end of its segment (segments that are not whole 64-row tiles) the rows
+    // beyond the end belong to the next expert, or to nobody: before the MMAs read the stage this thread clears
+    // them in the A operand (so that they add nothing), and after the last segment also in the B operand (rows
+    // nobody owns may hold anything, and 0 x NaN is not 0).
     if (lane == 0) {
       uint32_t it = 0, tile_iter = 0;
       int e = 0;
       bool ok = true;
+      const int rows_in_use = seg_begin[a.n_ffn];
       for (int L = blockIdx.x; L < total_tiles && ok; L += gridDim.x, ++tile_iter) {
         const TileInfo ti = decode(L, e);
         const uint32_t buf = tile_iter & 1u, tph = (tile_iter >> 1) & 1u;
@@ -203,6 +208,19 @@ bwd_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant_
           if (!mbar_wait(smem_u32(&bar_full[s]), ph, &abort_flag, 33, err_word)) { ok = false; break; }
           tc_fence_after();
           const uint32_t a_addr = ring + s * kStageBytes, b_addr = a_addr + kABytes;
+          if (MODE == WGRAD) {
+            const int valid = (ti.row_end - ti.row0) - kb * BK;  // k rows of this tile that belong to the segment
+            if (valid < BK) {
+              // a k row is one 128-byte line of every 64-column box: lines [valid, 64) of the boxes concerned
+              uint8_t* stage = smem_raw + (ring - smem_u32(smem_raw)) + s * kStageBytes;
+              const int boxes = ti.row_end >= rows_in_use ? 6 : 2;  // A only, or A and B
+              for (int box = 0; box < boxes; ++box) {
+                uint4* p = reinterpret_cast<uint4*>(stage + box * kBoxBytes + valid * 128);
+                for (int i = 0; i < (BK - valid) * 8; ++i) p[i] = make_uint4(0u, 0u, 0u, 0u);
+              }
+              asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> visible to the MMAs
+            }
+          }
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
             // 16 k: K-major = 32 bytes inside the swizzle row; MN-major = 16 rows of 128 bytes
@@ -409,13 +427,13 @@ cudaError_t launch_token_outer_tc(const Dims& d, const void* P, const void* Q, f
   return run<WGRAD>(sms, mP, mP, mQ, mQ, a, st);
 }
 
-// bf16 FFN backward on the tensor cores.  cudaErrorNotSupported when it does not apply (storage type, segments
-// that are not whole 64-row k tiles, shapes the tensor maps cannot describe): the caller then uses the FMA path.
+// bf16 FFN backward on the tensor cores.  cudaErrorNotSupported when it does not apply (storage type, shapes the
+// tensor maps cannot describe): the caller then uses the FMA path.
 cudaError_t launch_ffn_backward_tc(const Dims& d, const void* x_perm, const int32_t* offsets, const void* W_gate,
                                    const void* W_up, const void* W_down, const void* h, const void* dy_perm,
                                    void* gate_buf, void* up_buf, void* dx_perm, float* dW_gate, float* dW_up,
                                    float* dW_down, cudaStream_t st, const void* gate_in, const void* up_in) {
-  if (d.dtype != MOEPP_BF16 || d.row_align % 64 != 0) return cudaErrorNotSupported;
+  if (d.dtype != MOEPP_BF16) return cudaErrorNotSupported;
   if (d.T == 0 || d.n_ffn == 0 || d.M_cap == 0) return cudaErrorNotSupported;
   int dev = 0, sms = 0;
   cudaError_t err = cudaGetDevice(&dev);

@@ -84,12 +84,13 @@ def test_backward_first_layer_vanilla(oracle64):
     check_backward(oracle64, lt)
 
 
-@pytest.mark.parametrize("dtype", ["f32", "bf16"])
-def test_backward_several_tiles(oracle64, dtype):
-    """Several 64-row tiles per expert with ragged tails, all four expert kinds, padded segments."""
+@pytest.mark.parametrize("dtype,row_align", [("f32", 128), ("bf16", 128), ("bf16", 1), ("bf16", 8)])
+def test_backward_several_tiles(oracle64, dtype, row_align):
+    """Several 64-row tiles per expert with ragged tails, all four expert kinds; padded segments, and dense ones
+    whose last weight-gradient k tile reaches into the next expert's rows (cleared in shared memory)."""
     spec = W.LayerSpec(T=1900, D=264, F=392, n_ffn=5, n_zero=1, n_copy=1, n_const=2, top_k=2, dtype=dtype)
     lt = W.make_layer(spec, seed=3, with_prev=True, w_std=0.05)
-    check_backward(oracle64, lt, row_align=128, add_residual=1)
+    check_backward(oracle64, lt, row_align=row_align, add_residual=1)
 
 
 @pytest.mark.parametrize("seed", range(6))
@@ -298,19 +299,21 @@ def test_backward_no_tokens():
 
 
 def test_backward_tensor_core_path_matches_fma_path():
-    """At a size the oracle cannot cover in seconds: the tensor-core GEMMs (row_align 128) against the FMA kernels
-    (forced by flag) on the same forward state; both were checked against the oracle at smaller sizes above."""
+    """At a size the oracle cannot cover in seconds: the tensor-core GEMMs against the FMA kernels (forced by flag)
+    on the same forward state, with padded (128) and dense (1) segments; both paths were checked against the oracle
+    at smaller sizes above."""
     spec = W.LayerSpec(T=6000, D=1032, F=1416, n_ffn=6, n_zero=1, n_copy=1, n_const=1, top_k=2, dtype="bf16")
     lt = W.make_layer(spec, seed=5, with_prev=True, w_std=0.03)
     wd = B.weights_from_tensors(lt)
     x, prev = lt.x.cuda(), lt.prev.cuda()
     gen = torch.Generator().manual_seed(9)
     dy = torch.randn(spec.T, spec.D, generator=gen).to(x.dtype).cuda()
-    res = []
-    for flags in (0, B.FLAG_SIMT_FFN):
-        cfg = B.config_from_spec(spec, row_align=128, flags=flags)
-        res.append(gpu_backward(cfg, wd, x, prev, dy, None)[0])
-    for name in GRADS:
-        a, b = res[0][name], res[1][name]
-        scale = max(float(np.abs(b).max()), 1e-6)
-        assert float(np.abs(a - b).max()) / scale <= 1e-2, name
+    for row_align in (128, 1):
+        res = []
+        for flags in (0, B.FLAG_SIMT_FFN):
+            cfg = B.config_from_spec(spec, row_align=row_align, flags=flags)
+            res.append(gpu_backward(cfg, wd, x, prev, dy, None)[0])
+        for name in GRADS:
+            a, b = res[0][name], res[1][name]
+            scale = max(float(np.abs(b).max()), 1e-6)
+            assert float(np.abs(a - b).max()) / scale <= 1e-2, (name, row_align)
