@@ -98,6 +98,8 @@ WORKLOADS = {  # name -> (config key, layers)
     "cfg2": ("cfg2_bf16_8e", 1),
     "cfg5": ("cfg5_sweep", 1),  # with --tokens and --zc-share
     "2b": ("paper_2b_32p8e", 1),  # the paper's 2B/(32+8)E layer shape
+    "06b": ("paper_06b_8p4e", 1),  # 0.6B/(8+4)E
+    "1b": ("paper_1b_16p4e", 1),  # 1B/(16+4)E
 }
 
 

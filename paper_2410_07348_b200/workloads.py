@@ -73,6 +73,10 @@ CONFIGS = {
     # the paper's 2B/(32+8)E model (Table 2): hidden 768, intermediate 2048, 32 FFN + 1/1/6 zero-computation
     # experts; a second router shape (40 experts, 52 stacked rows)
     "paper_2b_32p8e": LayerSpec(T=32768, D=768, F=2048, n_ffn=32, n_zero=1, n_copy=1, n_const=6),
+    # the other two small models of Table 2 (same hidden and intermediate size, 1/1/2 zero-computation experts);
+    # the 7B/(16+4)E model (hidden 1536, intermediate 4096) has cfg3's sizes
+    "paper_06b_8p4e": LayerSpec(T=32768, D=768, F=2048, n_ffn=8, n_zero=1, n_copy=1, n_const=2),
+    "paper_1b_16p4e": LayerSpec(T=32768, D=768, F=2048, n_ffn=16, n_zero=1, n_copy=1, n_const=2),
 }
 CFG4_LAYERS = 4
 CFG5_ZC_SHARES = (0.0, 0.15, 0.30, 0.50, 0.75)

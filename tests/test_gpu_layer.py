@@ -147,6 +147,14 @@ def test_paper_2b_shape_32_plus_8_experts(oracle64):
     assert np.all(info["counts"] > 0)
 
 
+@pytest.mark.parametrize("name", ["paper_06b_8p4e", "paper_1b_16p4e"])
+def test_paper_small_model_shapes(oracle64, name):
+    """The 0.6B/(8+4)E and 1B/(16+4)E layers of Table 2 (hidden 768, intermediate 2048)."""
+    lt = W.make_config(name, gen_device="cuda", device="cuda")
+    info = check_layer(oracle64, lt, 96)
+    assert np.all(info["counts"] > 0)
+
+
 def test_cfg4_stack_of_four(oracle64):
     """Free-running 4-layer stack on all 32768 tokens; the oracle follows the same picks on a token sample."""
     spec = W.CONFIGS["cfg4_7b_stack"]
