@@ -56,10 +56,12 @@ __device__ __forceinline__ uint64_t make_smem_desc_mn(uint32_t addr) {
 
 struct TileInfo {
   int e, row0, row_end, m0, n0, kb_count;
+  int second;  // WGRAD with two products in one launch: this tile belongs to the second (A from tmA1, C = C2)
 };
 
 struct Args {
   void* C;                 // DX: bf16 [M_cap, Nout];  WGRAD: float [n_ffn, Mout, Nout]
+  float* C2;               // WGRAD: output of a second product P2^T Q sharing Q with the first (nullptr: none)
   __nv_bfloat16 *gate, *up;  // DH: dGate, dUp out
   const __nv_bfloat16 *gate_in, *up_in;  // DH: pre-activations in (may be the same buffers)
   const int32_t* offsets;
@@ -88,7 +90,8 @@ bwd_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const int NT = (a.Nout + BN - 1) / BN;
-  const int MT = (a.Mout + BM - 1) / BM;  // WGRAD
+  const int MT1 = (a.Mout + BM - 1) / BM;                        // WGRAD: m tiles of one product
+  const int MT = (MODE == WGRAD && a.C2 != nullptr) ? 2 * MT1 : MT1;  // ... of the launch
   const int KB = (a.Kd + BK - 1) / BK;    // DH, DX
   int32_t* const err_word = a.err_word;
 
@@ -135,13 +138,16 @@ bwd_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant_
     ti.row_end = en;
     if (MODE == WGRAD) {
       ti.row0 = b;
-      ti.m0 = (local % MT) * BM;
+      const int mt = local % MT;
+      ti.second = mt >= MT1 ? 1 : 0;
+      ti.m0 = (ti.second ? mt - MT1 : mt) * BM;
       ti.n0 = (local / MT) * BN;
       ti.kb_count = (en - b + BK - 1) / BK;
     } else {
       const int mt = (en - b + BM - 1) / BM;
       ti.row0 = b + (local % mt) * BM;
       ti.m0 = 0;
+      ti.second = 0;
       ti.n0 = (local / mt) * BN;
       ti.kb_count = (MODE == DX ? 2 : 1) * KB;
     }
@@ -153,8 +159,8 @@ bwd_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant_
     if (lane == 0) {
       asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA0) : "memory");
       asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB0) : "memory");
+      if (MODE != DH) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA1) : "memory");
       if (MODE == DX) {
-        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA1) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB1) : "memory");
       }
       uint32_t it = 0;
@@ -171,7 +177,8 @@ bwd_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant_
           if (MODE == WGRAD) {
             const int krow = ti.row0 + kb * BK;  // k runs over the expert's rows
 #pragma unroll
-            for (int j = 0; j < BM / 64; ++j) tma_load_2d(a_dst + j * kBoxBytes, &tmA0, ti.m0 + 64 * j, krow, full);
+            for (int j = 0; j < BM / 64; ++j)
+              tma_load_2d(a_dst + j * kBoxBytes, ti.second ? &tmA1 : &tmA0, ti.m0 + 64 * j, krow, full);
 #pragma unroll
             for (int j = 0; j < BN / 64; ++j) tma_load_2d(b_dst + j * kBoxBytes, &tmB0, ti.n0 + 64 * j, krow, full);
           } else {
@@ -264,7 +271,8 @@ bwd_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant_
         const int m = ti.m0 + q * 32 + lane;
         const bool row_ok = m < a.Mout;
         const bool empty = ti.kb_count == 0;  // an expert without rows: the accumulator was never written
-        float* crow = static_cast<float*>(a.C) + ((size_t)ti.e * a.Mout + (row_ok ? m : 0)) * a.Nout + ti.n0;
+        float* crow = (ti.second ? a.C2 : static_cast<float*>(a.C)) +
+                      ((size_t)ti.e * a.Mout + (row_ok ? m : 0)) * a.Nout + ti.n0;
 #pragma unroll 1
         for (int c = 0; c < BN; c += 16) {
           uint32_t r[16];
@@ -488,12 +496,11 @@ cudaError_t launch_ffn_backward_tc(const Dims& d, const void* x_perm, const int3
   a.Mout = 0; a.Nout = d.F; a.Kd = d.D;
   err = d.D <= 2048 ? run<DH, 8>(sms, mDyK, mDyK, mWdMN, mWdMN, a, st) : run<DH, 4>(sms, mDyK, mDyK, mWdMN, mWdMN, a, st);
   if (err != cudaSuccess) return err;
-  // 4. dW_gate[e] = dGate_e^T Xp_e, dW_up[e] = dUp_e^T Xp_e
+  // 4. dW_gate[e] = dGate_e^T Xp_e and dW_up[e] = dUp_e^T Xp_e in one launch (they share the Xp tiles)
   a.gate = nullptr; a.up = nullptr; a.Mout = d.F; a.Nout = d.D; a.Kd = 0;
-  a.C = dW_gate;
-  if ((err = run<WGRAD>(sms, mGateMN, mGateMN, mXpMN, mXpMN, a, st)) != cudaSuccess) return err;
-  a.C = dW_up;
-  if ((err = run<WGRAD>(sms, mUpMN, mUpMN, mXpMN, mXpMN, a, st)) != cudaSuccess) return err;
+  a.C = dW_gate; a.C2 = dW_up;
+  if ((err = run<WGRAD>(sms, mGateMN, mUpMN, mXpMN, mXpMN, a, st)) != cudaSuccess) return err;
+  a.C2 = nullptr;
   // 5. dXp = dGate W_gate + dUp W_up
   a.C = dx_perm; a.Mout = 0; a.Nout = d.D; a.Kd = d.F;
   return run<DX>(sms, mGateK, mUpK, mWgMN, mWuMN, a, st);
