@@ -118,7 +118,7 @@ cudaError_t launch_ffn_backward_simt(const Dims& d, const void* x_perm, const in
                                      float* dW_down, cudaStream_t st, const void* gate_in = nullptr,
                                      const void* up_in = nullptr);
 
-// The same on the tensor cores (bf16, segments of whole 64-row tiles); cudaErrorNotSupported otherwise.
+// The same on the tensor cores (bf16 storage); cudaErrorNotSupported otherwise.
 cudaError_t launch_ffn_backward_tc(const Dims& d, const void* x_perm, const int32_t* offsets, const void* W_gate,
                                    const void* W_up, const void* W_down, const void* h, const void* dy_perm,
                                    void* gate_buf, void* up_buf, void* dx_perm, float* dW_gate, float* dW_up,
