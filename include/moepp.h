@@ -280,6 +280,15 @@ moepp_status moepp_layer_backward(const moepp_config* cfg, const moepp_weights* 
                                   void* stream);
 
 /*
+ * dst[i, :] = src[row_index[i], :] for i < n_rows; a negative index gives a row of zeros.  Rows of row_elems elements
+ * of `dtype`, row size a multiple of 16 bytes, device pointers.  The paper has no counterpart: this is the row
+ * regrouping an expert-parallel deployment (Sec. 3.4: FFN experts spread over GPUs, zero-computation experts on
+ * every GPU) needs between the all-to-all exchange and the grouped FFN, see paper_2410_07348_b200/expert_parallel.py.
+ */
+moepp_status moepp_gather_rows(const void* src, const int32_t* row_index, int64_t n_rows, int32_t row_elems,
+                               int32_t dtype, void* dst, void* stream);
+
+/*
  * The stack of moepp_stack_forward in a form that can be differentiated, and its backward pass: a training
  * step's worth of the layer (the paper trains all layers jointly on the language-model loss plus beta times
  * the sum of the layers' Eq. 7 losses, Sec. 3.4; it prints no backward formulas).

@@ -27,7 +27,8 @@ EXPORTS = ("moepp_status_string", "moepp_workspace_bytes", "moepp_workspace_byte
            "moepp_stack_workspace_bytes", "moepp_stack_forward", "moepp_stack_workspace_bytes_host",
            "moepp_stack_forward_host", "moepp_balance_stats", "moepp_backward_workspace_bytes",
            "moepp_layer_backward", "moepp_balance_backward", "moepp_stack_train_workspace_bytes",
-           "moepp_stack_forward_train", "moepp_stack_backward_workspace_bytes", "moepp_stack_backward")
+           "moepp_stack_forward_train", "moepp_stack_backward_workspace_bytes", "moepp_stack_backward",
+           "moepp_gather_rows")
 STATIC_SCRATCH_BYTES = 32 << 20
 
 
@@ -203,6 +204,14 @@ def moepp_balance_stats(cfg, logits, expert_counts, f, P, loss):
     c = cfg.c()
     _check(lib().moepp_balance_stats(ctypes.byref(c), _p(logits), _p(expert_counts), _p(f), _p(P), _p(loss),
                                      _stream()), "moepp_balance_stats")
+
+
+def moepp_gather_rows(src, row_index, dst):
+    """dst[i, :] = src[row_index[i], :] (zeros for a negative index); src, dst: 2-D CUDA tensors of one dtype."""
+    assert src.dtype == dst.dtype and src.shape[1] == dst.shape[1] and row_index.dtype == torch.int32
+    dt = MOEPP_BF16 if src.dtype == torch.bfloat16 else MOEPP_F32
+    _check(lib().moepp_gather_rows(_p(src), _p(row_index), ctypes.c_int64(dst.shape[0]), ctypes.c_int32(src.shape[1]),
+                                   ctypes.c_int32(dt), _p(dst), _stream()), "moepp_gather_rows")
 
 
 def _grads(grads: dict) -> moepp_grads:

@@ -238,6 +238,16 @@ moepp_status moepp_permute(const moepp_config* cfg, const void* x, const int32_t
                                   static_cast<cudaStream_t>(stream)));
 }
 
+moepp_status moepp_gather_rows(const void* src, const int32_t* row_index, int64_t n_rows, int32_t row_elems,
+                               int32_t dtype, void* dst, void* stream) {
+  if (n_rows < 0 || row_elems <= 0 || (dtype != MOEPP_F32 && dtype != MOEPP_BF16)) return MOEPP_ERR_INVALID_ARG;
+  const size_t row_bytes = (size_t)row_elems * elem_size(dtype);
+  if (row_bytes % 16 != 0) return MOEPP_ERR_ALIGN;
+  if (n_rows > 0 && (src == nullptr || row_index == nullptr || dst == nullptr)) return MOEPP_ERR_INVALID_ARG;
+  if (!aligned16(src) || !aligned16(dst)) return MOEPP_ERR_ALIGN;
+  return from_cuda(launch_gather_rows(src, row_index, n_rows, row_bytes, dst, static_cast<cudaStream_t>(stream)));
+}
+
 moepp_status moepp_grouped_ffn(const moepp_config* cfg, const void* x_perm, const int32_t* expert_offsets,
                                const void* W_gate, const void* W_up, const void* W_down, void* h_ws, void* y_perm,
                                void* stream) {

@@ -41,6 +41,9 @@ cudaError_t launch_route_tc(const Dims& d, const void* x, const float* W_r, cons
 cudaError_t launch_permute(const Dims& d, const void* x, const int32_t* topk_idx, const int32_t* offsets,
                            int32_t* row_of_slot, int32_t* slot_of_row, void* x_perm, cudaStream_t st);
 
+cudaError_t launch_gather_rows(const void* src, const int32_t* index, long long n_rows, size_t row_bytes, void* dst,
+                               cudaStream_t st);
+
 // gate_out / up_out (both or neither): the SwiGLU pre-activations [M_cap, F] are stored as well
 cudaError_t launch_ffn_simt(const Dims& d, const void* x_perm, const int32_t* offsets, const void* W_gate,
                             const void* W_up, const void* W_down, void* h, void* y_perm, cudaStream_t st,

@@ -123,7 +123,37 @@ permute_gather_kernel(const XT* __restrict__ x, const int32_t* __restrict__ slot
   for (; i < nvec; i += 32) dst[i] = __ldg(src + i);
 }
 
+// dst[i, :] = src[index[i], :] (zeros where index[i] < 0); one warp per row, rows of `bytes` bytes (multiple of 16)
+__global__ void __launch_bounds__(256)
+gather_rows_kernel(const uint4* __restrict__ src, const int32_t* __restrict__ index, long long n_rows, int vec_per_row,
+                   uint4* __restrict__ dst) {
+  const int lane = threadIdx.x & 31;
+  const long long row = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= n_rows) return;
+  const int from = index[row];
+  uint4* d = dst + (size_t)row * vec_per_row;
+  if (from < 0) {
+    for (int i = lane; i < vec_per_row; i += 32) d[i] = make_uint4(0u, 0u, 0u, 0u);
+    return;
+  }
+  const uint4* s = src + (size_t)from * vec_per_row;
+  int i = lane;
+  for (; i + 96 < vec_per_row; i += 128) {  // four loads in flight per lane
+    const uint4 a = __ldg(s + i), b = __ldg(s + i + 32), c = __ldg(s + i + 64), e = __ldg(s + i + 96);
+    d[i] = a; d[i + 32] = b; d[i + 64] = c; d[i + 96] = e;
+  }
+  for (; i < vec_per_row; i += 32) d[i] = __ldg(s + i);
+}
+
 }  // namespace
+
+cudaError_t launch_gather_rows(const void* src, const int32_t* index, long long n_rows, size_t row_bytes, void* dst,
+                               cudaStream_t st) {
+  if (n_rows == 0) return cudaSuccess;
+  gather_rows_kernel<<<(unsigned)((n_rows + 7) / 8), 256, 0, st>>>(static_cast<const uint4*>(src), index, n_rows,
+                                                                  (int)(row_bytes / 16), static_cast<uint4*>(dst));
+  return cudaGetLastError();
+}
 
 cudaError_t launch_permute(const Dims& d, const void* x, const int32_t* topk_idx, const int32_t* offsets,
                            int32_t* row_of_slot, int32_t* slot_of_row, void* x_perm, cudaStream_t st) {
