@@ -31,7 +31,7 @@ import torch  # noqa: E402
 
 # DRAM bytes (read + write) of one grouped-FFN call (GEMM 1 + GEMM 2 launches), taken from an ncu capture of one
 # config-4 layer (dram__bytes_read.sum + dram__bytes_write.sum); only valid for the CTA-pair kernels on that shape.
-NCU_FFN_TRAFFIC_BYTES = {"cfg4": 2591.0e6}
+NCU_FFN_TRAFFIC_BYTES = {"cfg4": 2773.0e6}
 
 METRIC = "moepp_expert_forward_tokens_per_s"
 UNIT = "tokens/s"
