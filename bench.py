@@ -213,6 +213,8 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="use only the first N layers of the workload (profiling)")
     ap.add_argument("--flags", type=int, default=0, help="MOEPP_FLAG_* bits passed in the configuration")
     ap.add_argument("--no-backward", action="store_true", help="skip the backward-pass timing of layer 1")
+    ap.add_argument("--ep-emulate", type=int, default=0,
+                    help="also time the expert-parallel forward with this many ranks emulated on the one GPU")
     ap.add_argument("--backward-row-align", type=int, default=64, help="row_align of the backward-pass timings")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "moepp" else args.warmup
@@ -420,6 +422,31 @@ def main():
                              "balance_loss_per_layer": [float(v) for v in lb.cpu()]}
         del tws, sbw, glist
 
+    # ---- optional: the expert-parallel forward with all ranks emulated on this GPU (compute side only) -----------
+    ep = None
+    if args.ep_emulate > 1 and spec.n_ffn % args.ep_emulate == 0:
+        from paper_2410_07348_b200 import expert_parallel as EP
+        R = args.ep_emulate
+        n_loc = spec.n_ffn // R
+        cuts = [T * r // R for r in range(R + 1)]
+        ranks, xs_r, ps_r = [], [], []
+        for r in range(R):
+            sub = W.LayerSpec(cuts[r + 1] - cuts[r], spec.D, spec.F, spec.n_ffn, spec.n_zero, spec.n_copy, spec.n_const,
+                              spec.top_k, spec.dtype)
+            local = dict(wd)
+            for name in ("W_gate", "W_up", "W_down"):
+                local[name] = wd[name][r * n_loc:(r + 1) * n_loc]
+            ranks.append(EP.EpRank(r, R, B.config_from_spec(sub, add_residual=add_res, flags=args.flags), local, dev))
+            xs_r.append(x0[cuts[r]:cuts[r + 1]])
+            ps_r.append(None if p1 is None else p1[cuts[r]:cuts[r + 1]])
+        ms_ep, _ = timed(lambda: EP.forward_emulated(ranks, xs_r, ps_r), max(3, args.steps // 5), 3)
+        ep = {"ranks": R, "ms_all_ranks_on_one_gpu": ms_ep, "ms_per_rank": ms_ep / R,
+              "ms_single_gpu_layer_over_ranks": (ms_step / L) / R,
+              "what": "layer 1, every rank's phases run one after the other on this GPU, device copies in the place "
+                      "of the all-to-all: compute and local copies only, no interconnect time; includes one "
+                      "device-to-host read of the offsets and the host planning per rank"}
+        del ranks
+
     # ---- end to end through the host-buffer call --------------------------------------------------------------
     xh = x0.cpu().pin_memory()
     yh = torch.empty(T, spec.D, dtype=td).pin_memory()
@@ -474,6 +501,7 @@ def main():
                     "speedup_of_moepp": ms_van / ms_step,
                     "what": "same library, same T, D, F, n_ffn, K, no zero-computation experts"},
         "backward": bwd,
+        "expert_parallel_emulated": ep,
         "cpu_baseline": cpu,
         "paper_context": "paper reports 1.1-2.1x expert forward throughput over vanilla MoE (A100 cluster, conditions "
                          "unstated); context only",
